@@ -1,0 +1,306 @@
+"""CPU oracle for the online hot path of TCA-Attention (test infrastructure).
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, fp64 NumPy restatement of what the
+paper defines; it shares no code with the CUDA library, is never imported by the
+product path, and exists so that the kernels have something independent to be compared
+against.  Only the tests, the smoke check and the benchmark's CPU-baseline leg call it.
+
+Inputs are the exact values the GPU sees (bf16 inputs are rounded to bf16 first and then
+widened to fp64 by the caller).  Token indices are 0-based (the paper is 1-based).
+
+Notation (Section 4 of the paper): L sequence length, d_h head dimension, b block size,
+w local window, m number of blocks, K = {1, 2, 4, ..., b} per-block retain counts,
+p the per-head configuration over K, s the token importance, h the block metric,
+Psi the budget map, t the per-block requirement, S the selected index set.
+
+Readings taken where the paper is silent or ambiguous (each is listed in the design
+notes with its justification):
+  * causal mask; the local subset is the w most recent tokens *of each query*;
+  * candidates for the global subset are [0, m*b) with m = floor((L - w) / b); the rest,
+    R = [m*b, L), is always kept (so global and local never overlap at the last query
+    and a 100 % budget is exactly dense causal attention);
+  * s is normalised over all L keys (Eq. 5 literally);
+  * grouped-query attention: one selection per KV head from the mean of the group's
+    per-query-head softmax distributions;
+  * larger h => larger retain count: blocks ranked ascending by (h, block index) and
+    Psi listed ascending (Eq. 7);
+  * the run lengths of Psi are floor(m * p_k) plus a largest-remainder correction so
+    that Psi has exactly m entries;
+  * ties inside Top(t; B) go to the lower token index;
+  * decoding: the block that leaves the window is the one compressed.
+
+Parity pins (tests/test_oracle_pins.py): dense causal attention by an independent
+brute force at 100 % budget and at w >= L; masked attention against an independently
+built boolean mask; closed forms of the concentration term; a hand-worked selection
+example; the exact identity ||s - s~||_1 = 2*gamma behind Theorem 1; decode == last
+prefill row; invariants of the selection.  "Parity unpinned" against the authors' own
+implementation: GQA aggregation, the window/partition reading, the leftover rounding
+and the decode block choice -- the paper fixes none of them; they are pinned only to
+the readings above.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+__all__ = [
+    "retain_counts", "num_blocks", "log_importance", "block_metric", "resolve_counts",
+    "budget_map", "mean_retain_floor", "rank_blocks", "block_requirement",
+    "select_tokens", "retained_set", "select_head", "visible_mask_row",
+    "attention_rows", "attention_over_set", "candidate_grid", "DecodeCache",
+    "dropped_mass",
+]
+
+
+# ----------------------------------------------------------------------------- helpers
+def _logsumexp(x: np.ndarray, axis=None) -> np.ndarray:
+    mx = np.max(x, axis=axis, keepdims=True)
+    out = mx + np.log(np.sum(np.exp(x - mx), axis=axis, keepdims=True))
+    return np.squeeze(out, axis=axis) if axis is not None else float(out.reshape(()))
+
+
+def retain_counts(b: int) -> np.ndarray:
+    """The set K = {1, 2, 4, ..., b} (Section 4.1)."""
+    if b < 1 or (b & (b - 1)):
+        raise ValueError("block size must be a power of two")
+    return 2 ** np.arange(int(b).bit_length(), dtype=np.int64)
+
+
+def num_blocks(L: int, b: int, w: int) -> int:
+    """m: number of candidate blocks; tokens [m*b, L) form the always-kept tail.
+
+    Section 4.2 partitions the sequence into blocks of b and puts what does not divide
+    into the local subset; with the no-overlap requirement of Section 4 the candidates
+    are the tokens outside the last query's window.
+    """
+    return max(0, (L - w) // b)
+
+
+# ----------------------------------------------------------------------------- step 1: Eq. 5
+def log_importance(q_last: np.ndarray, K: np.ndarray, sm_scale: float) -> np.ndarray:
+    """log s for one KV head.  q_last: [G, d] (the group's last-token queries), K: [L, d].
+
+    Eq. 5: s = softmax(q_L K^T / sqrt(d_h)) over all L keys, for each query head of the
+    group; the group's distributions are averaged (a probability vector again).  The
+    logarithm is returned because s underflows for long sequences.
+    """
+    q_last = np.atleast_2d(np.asarray(q_last, dtype=np.float64))
+    K = np.asarray(K, dtype=np.float64)
+    x = (q_last @ K.T) * sm_scale                       # [G, L] logits
+    logp = x - _logsumexp(x, axis=1)[:, None]           # per-query-head log-softmax
+    return _logsumexp(logp, axis=0) - math.log(q_last.shape[0])
+
+
+# ----------------------------------------------------------------------------- step 2-3: Eq. 6
+def block_metric(log_s: np.ndarray, m: int, b: int, alpha: float) -> np.ndarray:
+    """h_j of Eq. 6 for blocks j < m, from log s.
+
+    h_j = (1 - alpha) * sum_i s_i + alpha * (1 - sum_i s_i^2 / (sum_i s_i)^2).
+    The second term is invariant to a common scale of the block's scores, so it is
+    evaluated on s_i / max_i s_i, which never divides zero by zero.
+    """
+    h = np.empty(m, dtype=np.float64)
+    for j in range(m):
+        l = np.asarray(log_s[j * b:(j + 1) * b], dtype=np.float64)
+        top = float(np.max(l))
+        e = np.exp(l - top)
+        mass = math.exp(top) * float(np.sum(e))
+        concentration = 1.0 - float(np.sum(e * e)) / float(np.sum(e)) ** 2
+        h[j] = (1.0 - alpha) * mass + alpha * concentration
+    return h
+
+
+# ----------------------------------------------------------------------------- step 4: Eq. 7
+def resolve_counts(p: Sequence[float], m: int) -> np.ndarray:
+    """n_k: how many of the m blocks get retain count k, k in K ascending.
+
+    Eq. 7 uses floor(m * p_k), which can leave Psi shorter than m; the shortfall D is
+    given, one each, to the D entries with the largest fractional part of m * p_k
+    (ties to the larger k).
+    """
+    p = np.asarray(p, dtype=np.float64)
+    if abs(float(p.sum()) - 1.0) > 1e-9 or np.any(p < 0):
+        raise ValueError("configuration must be a probability vector")
+    f = m * p
+    n = np.floor(f).astype(np.int64)
+    short = int(m - n.sum())
+    frac = f - n
+    order = sorted(range(len(p)), key=lambda k: (-frac[k], -k))
+    for k in order[:short]:
+        n[k] += 1
+    assert int(n.sum()) == m
+    return n
+
+
+def budget_map(n: Sequence[int], b: int) -> np.ndarray:
+    """Psi of Eq. 7: n_1 ones, n_2 twos, ..., n_b copies of b, in ascending order."""
+    ks = retain_counts(b)
+    return np.repeat(ks, np.asarray(n, dtype=np.int64))
+
+
+def mean_retain_floor(p: Sequence[float], b: int) -> int:
+    """t = floor(sum_k k * p_k): tokens kept from a block completed while decoding."""
+    return int(math.floor(float(np.dot(retain_counts(b).astype(np.float64),
+                                       np.asarray(p, dtype=np.float64)))))
+
+
+def rank_blocks(h: np.ndarray) -> np.ndarray:
+    """rank_j = position of block j when blocks are sorted ascending by (h_j, j)."""
+    order = np.lexsort((np.arange(len(h)), np.asarray(h, dtype=np.float64)))
+    rank = np.empty(len(h), dtype=np.int64)
+    rank[order] = np.arange(len(h))
+    return rank
+
+
+def block_requirement(h: np.ndarray, n: Sequence[int], b: int) -> np.ndarray:
+    """t_j = Psi[rank_j] (Eq. 7): the densest blocks get the largest retain counts."""
+    psi = budget_map(n, b)
+    return psi[rank_blocks(h)]
+
+
+# ----------------------------------------------------------------------------- step 5: Eq. 8
+def select_tokens(log_s: np.ndarray, t: Sequence[int], b: int) -> np.ndarray:
+    """S = union_j Top(t_j; B_j) by s (Eq. 8), ascending.  Ties: lower index wins."""
+    keep: List[int] = []
+    for j, tj in enumerate(t):
+        blk = np.asarray(log_s[j * b:(j + 1) * b], dtype=np.float64)
+        order = np.argsort(-blk, kind="stable")         # stable => lower index first on ties
+        keep.extend(int(j * b + i) for i in order[:int(tj)])
+    return np.array(sorted(keep), dtype=np.int64)
+
+
+def retained_set(S: np.ndarray, m: int, b: int, L: int) -> np.ndarray:
+    """T = S union [m*b, L): everything the cache keeps after prefilling."""
+    return np.concatenate([np.asarray(S, dtype=np.int64), np.arange(m * b, L, dtype=np.int64)])
+
+
+def select_head(q_last, K, p, b: int, w: int, alpha: float, sm_scale: float):
+    """Steps 1-6 of Algorithm 2 for one KV head.  Returns a dict of every intermediate."""
+    L = K.shape[0]
+    m = num_blocks(L, b, w)
+    log_s = log_importance(q_last, K, sm_scale)
+    h = block_metric(log_s, m, b, alpha)
+    n = resolve_counts(p, m)
+    t = block_requirement(h, n, b)
+    S = select_tokens(log_s, t, b)
+    return {"log_s": log_s, "m": m, "h": h, "n": n, "t": t, "S": S,
+            "T": retained_set(S, m, b, L)}
+
+
+# ----------------------------------------------------------------------------- step 7: Eq. 2
+def visible_mask_row(i: int, T: np.ndarray, w: int, L: int) -> np.ndarray:
+    """Boolean [L]: keys query i attends to = {j <= i : j in T or i - j < w}."""
+    vis = np.zeros(L, dtype=bool)
+    vis[np.asarray(T, dtype=np.int64)] = True
+    lo = max(0, i - w + 1)
+    vis[lo:i + 1] = True
+    vis[i + 1:] = False
+    return vis
+
+
+def attention_over_set(q: np.ndarray, Ksel: np.ndarray, Vsel: np.ndarray, sm_scale: float) -> np.ndarray:
+    """softmax(q Ksel^T * scale) Vsel for one query vector (Eq. 2 for one row)."""
+    x = (np.asarray(Ksel, dtype=np.float64) @ np.asarray(q, dtype=np.float64)) * sm_scale
+    x -= x.max()
+    e = np.exp(x)
+    return (e / e.sum()) @ np.asarray(Vsel, dtype=np.float64)
+
+
+def attention_rows(Q: np.ndarray, K: np.ndarray, V: np.ndarray, T: np.ndarray, w: int,
+                   sm_scale: float, rows: Optional[Sequence[int]] = None) -> np.ndarray:
+    """Sparse causal attention (Eq. 2) for one query head: rows of Q -> [len(rows), d].
+
+    Query i attends to [K^G; K^L] = keys {j <= i : j in T} plus its own last w keys,
+    taken as a set.
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    L = K.shape[0]
+    rows = range(Q.shape[0]) if rows is None else rows
+    out = np.empty((len(rows), V.shape[1]), dtype=np.float64)
+    for r, i in enumerate(rows):
+        vis = visible_mask_row(int(i), T, w, L)
+        out[r] = attention_over_set(Q[int(i)], K[vis], V[vis], sm_scale)
+    return out
+
+
+def dropped_mass(q: np.ndarray, K: np.ndarray, i: int, T: np.ndarray, w: int, sm_scale: float) -> float:
+    """gamma_i of Theorem 1: dense-softmax mass of the causally visible keys not kept."""
+    L = K.shape[0]
+    x = (np.asarray(K[:i + 1], dtype=np.float64) @ np.asarray(q, dtype=np.float64)) * sm_scale
+    x -= x.max()
+    e = np.exp(x)
+    vis = visible_mask_row(i, T, w, L)[:i + 1]
+    return float(e[~vis].sum() / e.sum())
+
+
+# ----------------------------------------------------------------------------- Eq. 3
+def candidate_grid(b: int, M: int = 14, sigma: float = 1.0) -> np.ndarray:
+    """The M log-Gaussian candidate configurations of Eq. 3, [M, |K|].
+
+    mu^i = log2(1 + (i - 1)(b - 1)/(M - 1)), i = 1..M;  p_k ~ exp(-(log2 k - mu)^2 / 2 sigma^2).
+    """
+    x = np.log2(retain_counts(b).astype(np.float64))
+    rows = []
+    for i in range(1, M + 1):
+        mu = math.log2(1.0 + (i - 1) * (b - 1) / (M - 1))
+        phi = np.exp(-((x - mu) ** 2) / (2.0 * sigma * sigma))
+        rows.append(phi / phi.sum())
+    return np.stack(rows)
+
+
+# ----------------------------------------------------------------------------- steps 8-9: decoding
+@dataclass
+class DecodeCache:
+    """Retained cache of one KV head while decoding (Section 4.2, last paragraph).
+
+    ``glob`` holds positions of the global subset, ``tail`` the always-kept recent
+    tokens.  After a token is appended, when the tail holds w + b tokens its oldest b
+    form a new block: they are scored with the current query (Eq. 5 restricted to the
+    block: each query head's softmax is taken over the block's b keys and the group's
+    distributions are averaged; with one query head the normaliser cannot change the
+    order), the top t = floor(sum_k k p_k) are moved to the global subset and the rest
+    dropped.
+    """
+    b: int
+    w: int
+    t_keep: int
+    sm_scale: float
+    glob: List[int] = field(default_factory=list)
+    tail: List[int] = field(default_factory=list)
+
+    @classmethod
+    def from_prefill(cls, S: np.ndarray, m: int, L: int, b: int, w: int, p, sm_scale: float) -> "DecodeCache":
+        return cls(b=b, w=w, t_keep=mean_retain_floor(p, b), sm_scale=sm_scale,
+                   glob=[int(x) for x in S], tail=list(range(m * b, L)))
+
+    def positions(self) -> np.ndarray:
+        return np.array(self.glob + self.tail, dtype=np.int64)
+
+    def append(self, pos: int, q_cur: np.ndarray, K_all: np.ndarray) -> Optional[np.ndarray]:
+        """Append token ``pos``; compress if a block completed.  q_cur: [G, d] queries of
+        the current token, K_all: keys indexable by position.  Returns the kept positions
+        of the compressed block, or None."""
+        self.tail.append(int(pos))
+        if len(self.tail) < self.w + self.b:
+            return None
+        blk = self.tail[:self.b]
+        self.tail = self.tail[self.b:]
+        q_cur = np.atleast_2d(np.asarray(q_cur, dtype=np.float64))
+        x = (q_cur @ np.asarray(K_all[blk], dtype=np.float64).T) * self.sm_scale   # [G, b]
+        # group mean of softmax restricted to the block, in the log domain
+        logp = x - _logsumexp(x, axis=1)[:, None]
+        score = _logsumexp(logp, axis=0)
+        order = np.argsort(-score, kind="stable")[:self.t_keep]
+        kept = sorted(blk[i] for i in order)
+        self.glob.extend(kept)
+        return np.array(kept, dtype=np.int64)
+
+    def attend(self, q: np.ndarray, K_all: np.ndarray, V_all: np.ndarray) -> np.ndarray:
+        """One decode step for one query head: attention over the whole retained cache."""
+        pos = self.positions()
+        return attention_over_set(q, K_all[pos], V_all[pos], self.sm_scale)

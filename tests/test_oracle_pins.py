@@ -1,0 +1,369 @@
+"""Pins for the CPU oracle: values and identities fixed by the paper and by mathematics.
+
+None of these tests touches the CUDA path.  Each one is chosen so that a plausible
+mistake in the oracle (dropped term, wrong sign, wrong index, transposed operand, wrong
+sort direction, off-by-one in the window) makes it fail.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+from scipy.special import softmax as sp_softmax
+
+from oracle import tca_oracle as O
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+# ----------------------------------------------------------------------------- brute force used as pins
+def dense_causal_attention(Q, K, V, scale):
+    """Textbook causal softmax attention on the full L x L matrix (library softmax)."""
+    L = K.shape[0]
+    A = (Q @ K.T) * scale
+    A = np.where(np.tril(np.ones((L, L), dtype=bool)), A, -np.inf)
+    return sp_softmax(A, axis=1) @ V
+
+
+def masked_attention_by_definition(Q, K, V, T, w, scale):
+    """Attention with a boolean mask written out from the set definition, entry by entry."""
+    L = K.shape[0]
+    Tset = set(int(x) for x in T)
+    mask = np.zeros((L, L), dtype=bool)
+    for i in range(L):
+        for j in range(L):
+            mask[i, j] = (j <= i) and ((j in Tset) or (i - j < w))
+    A = np.where(mask, (Q @ K.T) * scale, -np.inf)
+    return sp_softmax(A, axis=1) @ V
+
+
+# ----------------------------------------------------------------------------- Eq. 5: importance
+def test_importance_is_a_distribution_and_matches_closed_form():
+    rng = _rng(1)
+    d, L = 16, 200
+    u = rng.standard_normal(d)
+    c = rng.standard_normal(L) * 3
+    K = c[:, None] * u[None, :]                     # k_j = c_j u, q = u  =>  logit_j = c_j |u|^2 scale
+    scale = 1 / math.sqrt(d)
+    ls = O.log_importance(u[None, :], K, scale)
+    assert abs(np.exp(ls).sum() - 1) < 1e-12
+    want = sp_softmax(c * (u @ u) * scale)
+    np.testing.assert_allclose(np.exp(ls), want, rtol=1e-11, atol=0)
+
+
+def test_importance_uses_the_scale_and_is_shift_invariant():
+    rng = _rng(2)
+    d, L = 8, 64
+    q = rng.standard_normal((1, d))
+    K = rng.standard_normal((L, d))
+    a = O.log_importance(q, K, 0.5)
+    # adding the same vector to every key adds a constant to every logit
+    b = O.log_importance(q, K + rng.standard_normal(d)[None, :], 0.5)
+    np.testing.assert_allclose(a, b, atol=1e-12)
+    # doubling the scale equals doubling the query
+    np.testing.assert_allclose(O.log_importance(q, K, 1.0), O.log_importance(2 * q, K, 0.5), atol=1e-12)
+    assert np.max(np.abs(O.log_importance(q, K, 1.0) - a)) > 1e-3
+
+
+def test_importance_group_mean_is_mean_of_softmaxes():
+    rng = _rng(3)
+    G, d, L = 4, 8, 50
+    q = rng.standard_normal((G, d))
+    K = rng.standard_normal((L, d))
+    want = np.mean([sp_softmax((K @ q[g]) * 0.3) for g in range(G)], axis=0)
+    np.testing.assert_allclose(np.exp(O.log_importance(q, K, 0.3)), want, rtol=1e-12)
+
+
+def test_importance_survives_underflow():
+    # logits far apart: probabilities underflow in fp64 but their logs must not
+    K = np.array([[0.0], [-2000.0], [-4000.0]])
+    ls = O.log_importance(np.array([[1.0]]), K, 1.0)
+    np.testing.assert_allclose(ls, [0.0, -2000.0, -4000.0], atol=1e-9)
+
+
+# ----------------------------------------------------------------------------- Eq. 6: block metric
+@pytest.mark.parametrize("b", [4, 32, 128])
+def test_block_metric_closed_forms(b):
+    alpha = 0.3
+    # uniform block: mass b*c, concentration 1 - 1/b
+    c = 1e-3
+    h = O.block_metric(np.log(np.full(b, c)), 1, b, alpha)[0]
+    assert h == pytest.approx((1 - alpha) * b * c + alpha * (1 - 1 / b), rel=1e-13)
+    # all mass on one token: concentration 0 (other tokens underflow to nothing)
+    ls = np.full(b, -5000.0)
+    ls[b // 2] = math.log(0.25)
+    h = O.block_metric(ls, 1, b, alpha)[0]
+    assert h == pytest.approx((1 - alpha) * 0.25, rel=1e-13)
+    # two equal tokens: concentration 1/2
+    ls = np.full(b, -5000.0)
+    ls[0] = ls[-1] = math.log(0.1)
+    h = O.block_metric(ls, 1, b, alpha)[0]
+    assert h == pytest.approx((1 - alpha) * 0.2 + alpha * 0.5, rel=1e-13)
+
+
+def test_block_metric_weights_and_scale_invariance():
+    rng = _rng(4)
+    b, m = 8, 3
+    ls = np.log(rng.random(m * b) * 0.01)
+    h0 = O.block_metric(ls, m, b, 0.0)              # alpha = 0: mass only
+    np.testing.assert_allclose(h0, np.exp(ls).reshape(m, b).sum(1), rtol=1e-13)
+    h1 = O.block_metric(ls, m, b, 1.0)              # alpha = 1: concentration only
+    h1s = O.block_metric(ls - 7.0, m, b, 1.0)       # common scale leaves it unchanged
+    np.testing.assert_allclose(h1, h1s, rtol=1e-12)
+    assert np.all(h1 > 0) and np.all(h1 < 1 - 1 / b + 1e-12)
+    # an empty-looking block (everything underflows) is still finite
+    assert np.isfinite(O.block_metric(np.full(b, -1e5), 1, b, 0.5)[0])
+
+
+# ----------------------------------------------------------------------------- Eq. 7: budget map
+def test_resolve_counts_hand_case_and_invariants():
+    np.testing.assert_array_equal(O.resolve_counts([0.5, 0.3, 0.2], 5), [2, 2, 1])
+    np.testing.assert_array_equal(O.budget_map([2, 2, 1], 4), [1, 1, 2, 2, 4])
+    assert O.mean_retain_floor([0.5, 0.3, 0.2], 4) == 1          # floor(1.9)
+    rng = _rng(5)
+    for _ in range(200):
+        nK = int(rng.integers(1, 9))
+        p = rng.dirichlet(np.ones(nK))
+        m = int(rng.integers(0, 2000))
+        n = O.resolve_counts(p, m)
+        assert n.sum() == m and np.all(n >= 0)
+        assert np.all(np.abs(n - m * p) < 1.0)
+        assert np.all(n >= np.floor(m * p))
+    # exact products need no correction
+    np.testing.assert_array_equal(O.resolve_counts([0.25, 0.75], 8), [2, 6])
+    with pytest.raises(ValueError):
+        O.resolve_counts([0.5, 0.4], 10)
+
+
+def test_budget_map_is_ascending_and_one_per_block():
+    psi = O.budget_map([3, 0, 2, 1], 8)
+    np.testing.assert_array_equal(psi, [1, 1, 1, 4, 4, 8])
+
+
+def test_rank_is_ascending_with_index_tiebreak():
+    h = np.array([0.3, 0.1, 0.3, 0.2, 0.1])
+    np.testing.assert_array_equal(O.rank_blocks(h), [3, 0, 4, 2, 1])
+    # densest block gets the largest count
+    t = O.block_requirement(np.array([0.9, 0.1, 0.5]), [1, 1, 1], 4)
+    np.testing.assert_array_equal(t, [4, 1, 2])
+
+
+# ----------------------------------------------------------------------------- hand-worked example
+def test_hand_worked_selection(golden):
+    g = golden("hand_selection.txt")
+    b, w, L, alpha = int(g["block"][0]), int(g["window"][0]), int(g["length"][0]), g["alpha"][0]
+    s = np.array(g["s"])
+    assert len(s) == L and abs(s.sum() - 1) < 1e-12
+    m = O.num_blocks(L, b, w)
+    assert m == int(g["m"][0])
+    ls = np.log(s)
+    np.testing.assert_allclose(O.block_metric(ls, m, b, 0.0), g["mass"], rtol=1e-12)
+    np.testing.assert_allclose(O.block_metric(ls, m, b, 1.0), g["concentration"], rtol=1e-12)
+    h = O.block_metric(ls, m, b, alpha)
+    np.testing.assert_allclose(h, g["h"], rtol=1e-12)
+    n = O.resolve_counts(g["p"], m)
+    np.testing.assert_array_equal(n, np.array(g["n"], dtype=int))
+    np.testing.assert_array_equal(O.budget_map(n, b), np.array(g["psi"], dtype=int))
+    np.testing.assert_array_equal(O.rank_blocks(h), np.array(g["rank"], dtype=int))
+    t = O.block_requirement(h, n, b)
+    np.testing.assert_array_equal(t, np.array(g["t"], dtype=int))
+    S = O.select_tokens(ls, t, b)
+    np.testing.assert_array_equal(S, np.array(g["S"], dtype=int))
+    np.testing.assert_array_equal(O.retained_set(S, m, b, L), np.array(g["T"], dtype=int))
+    assert O.mean_retain_floor(g["p"], b) == int(g["t_decode"][0])
+
+
+# ----------------------------------------------------------------------------- Eq. 8: top-t
+def test_top_t_is_the_best_subset_by_brute_force():
+    rng = _rng(6)
+    b = 8
+    for _ in range(30):
+        ls = rng.standard_normal(b)
+        for t in (1, 2, 4, 8):
+            S = O.select_tokens(ls, [t], b)
+            best = max(itertools.combinations(range(b), t), key=lambda c: sum(ls[list(c)]))
+            assert sorted(best) == list(S)
+
+
+def test_top_t_ties_go_to_lower_index_and_output_sorted():
+    ls = np.log(np.array([.1, .3, .3, .1, .3, .1, .1, .1]))
+    np.testing.assert_array_equal(O.select_tokens(ls, [2], 8), [1, 2])
+    np.testing.assert_array_equal(O.select_tokens(ls, [4], 8), [0, 1, 2, 4])
+    # second block is offset by b
+    two = np.concatenate([ls, ls])
+    np.testing.assert_array_equal(O.select_tokens(two, [1, 2], 8), [1, 9, 10])
+
+
+def test_selection_invariants_on_random_heads():
+    rng = _rng(7)
+    b, w, L, d, G = 16, 40, 40 + 16 * 9 + 5, 8, 2
+    for trial in range(5):
+        K = rng.standard_normal((L, d))
+        q = rng.standard_normal((G, d))
+        p = rng.dirichlet(np.ones(5))
+        r = O.select_head(q, K, p, b, w, 0.5, 0.35)
+        m, S, t, h, n = r["m"], r["S"], r["t"], r["h"], r["n"]
+        assert m == 9
+        ks = O.retain_counts(b)
+        assert len(S) == int((ks * n).sum())
+        assert np.all(np.diff(S) > 0) and S.max() < m * b
+        np.testing.assert_array_equal(np.bincount(S // b, minlength=m), t)
+        np.testing.assert_array_equal(np.sort(t), O.budget_map(n, b))
+        for a in range(m):
+            for c in range(m):
+                if h[a] < h[c]:
+                    assert t[a] <= t[c]
+        for j in range(m):
+            blk = r["log_s"][j * b:(j + 1) * b]
+            kept = np.zeros(b, bool)
+            kept[S[(S // b) == j] - j * b] = True
+            if kept.any() and (~kept).any():
+                assert blk[kept].min() >= blk[~kept].max()
+        # tail [m*b, L) always kept, once
+        T = r["T"]
+        assert len(set(T.tolist())) == len(T)
+        np.testing.assert_array_equal(T[len(S):], np.arange(m * b, L))
+
+
+# ----------------------------------------------------------------------------- Eq. 2: attention
+def _toy(seed, L=96, d=8):
+    rng = _rng(seed)
+    return (rng.standard_normal((L, d)), rng.standard_normal((L, d)) * 1.5,
+            rng.standard_normal((L, d)))
+
+
+def test_full_budget_is_dense_causal_attention():
+    Q, K, V = _toy(8)
+    L, d = K.shape
+    b, w, scale = 8, 24, 1 / math.sqrt(d)
+    nK = int(b).bit_length()
+    p = np.zeros(nK)
+    p[-1] = 1.0                                       # every block keeps all b tokens
+    r = O.select_head(Q[-1:], K, p, b, w, 0.5, scale)
+    np.testing.assert_array_equal(r["T"], np.arange(L))
+    got = O.attention_rows(Q, K, V, r["T"], w, scale)
+    np.testing.assert_allclose(got, dense_causal_attention(Q, K, V, scale), rtol=1e-11, atol=1e-13)
+
+
+def test_window_covering_everything_is_dense_causal_attention():
+    Q, K, V = _toy(9, L=50)
+    scale = 0.4
+    p = np.array([1.0, 0, 0, 0])                       # would keep 1 per block, but there are no blocks
+    r = O.select_head(Q[-1:], K, p, 8, 64, 0.5, scale)
+    assert r["m"] == 0 and len(r["S"]) == 0
+    got = O.attention_rows(Q, K, V, r["T"], 64, scale)
+    np.testing.assert_allclose(got, dense_causal_attention(Q, K, V, scale), rtol=1e-11, atol=1e-13)
+
+
+@pytest.mark.parametrize("w", [1, 5, 16])
+def test_sparse_attention_matches_mask_written_from_the_definition(w):
+    Q, K, V = _toy(10, L=70)
+    scale = 0.37
+    b = 4
+    p = np.array([0.6, 0.3, 0.1])
+    r = O.select_head(Q[-1:], K, p, b, w, 0.5, scale)
+    got = O.attention_rows(Q, K, V, r["T"], w, scale)
+    want = masked_attention_by_definition(Q, K, V, r["T"], w, scale)
+    np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-13)
+    # it really is sparse: differs from dense attention somewhere
+    assert np.max(np.abs(got - dense_causal_attention(Q, K, V, scale))) > 1e-4
+
+
+def test_error_identity_and_bound_of_theorem_1():
+    Q, K, V = _toy(11, L=80)
+    scale, b, w = 0.5, 8, 16
+    p = np.array([0.5, 0.3, 0.2, 0.0])
+    r = O.select_head(Q[-1:], K, p, b, w, 0.5, scale)
+    dense = dense_causal_attention(Q, K, V, scale)
+    sparse = O.attention_rows(Q, K, V, r["T"], w, scale)
+    L = K.shape[0]
+    saw_drop = False
+    for i in range(L):
+        gamma = O.dropped_mass(Q[i], K, i, r["T"], w, scale)
+        vis = O.visible_mask_row(i, r["T"], w, L)
+        x = (K[:i + 1] @ Q[i]) * scale
+        s_full = sp_softmax(x)
+        s_kept = np.zeros(i + 1)
+        s_kept[vis[:i + 1]] = sp_softmax(x[vis[:i + 1]])
+        # exact identity behind the theorem: total variation is twice the dropped mass
+        assert abs(np.abs(s_full - s_kept).sum() - 2 * gamma) < 1e-12
+        err = dense[i] - sparse[i]
+        assert np.max(np.abs(err)) <= 2 * gamma * np.max(np.abs(V)) + 1e-12
+        assert np.sum(np.abs(err)) <= 2 * gamma * np.max(np.abs(V).sum(1)) + 1e-12
+        saw_drop |= gamma > 1e-6
+    assert saw_drop
+
+
+# ----------------------------------------------------------------------------- decoding
+def test_decode_over_retained_cache_equals_last_prefill_row():
+    Q, K, V = _toy(12, L=90)
+    scale, b, w = 0.45, 8, 20
+    p = np.array([0.4, 0.3, 0.2, 0.1])
+    r = O.select_head(Q[-1:], K, p, b, w, 0.5, scale)
+    L = K.shape[0]
+    cache = O.DecodeCache.from_prefill(r["S"], r["m"], L, b, w, p, scale)
+    np.testing.assert_array_equal(cache.positions(), r["T"])
+    last = O.attention_rows(Q, K, V, r["T"], w, scale, rows=[L - 1])[0]
+    np.testing.assert_allclose(cache.attend(Q[L - 1], K, V), last, rtol=1e-12, atol=1e-14)
+
+
+def test_decode_append_keeps_partition_and_compresses_the_block_leaving_the_window():
+    rng = _rng(13)
+    b, w, d = 8, 16, 8
+    L0, steps = 16 + 8 * 3, 30
+    K = rng.standard_normal((L0 + steps, d))
+    Qd = rng.standard_normal((L0 + steps, d))
+    p = np.array([0.1, 0.2, 0.3, 0.4])                # mean retain = .1+.4+1.2+3.2 = 4.9 -> 4
+    r = O.select_head(Qd[L0 - 1:L0], K[:L0], p, b, w, 0.5, 0.4)
+    cache = O.DecodeCache.from_prefill(r["S"], r["m"], L0, b, w, p, 0.4)
+    assert cache.t_keep == 4
+    n_glob = len(cache.glob)
+    for s in range(steps):
+        pos = L0 + s
+        kept = cache.append(pos, Qd[pos:pos + 1], K)
+        m_now = O.num_blocks(pos + 1, b, w)
+        # same partition as a prefill of length pos+1 would use
+        assert cache.tail == list(range(m_now * b, pos + 1))
+        assert w <= len(cache.tail) < w + b
+        if kept is not None:
+            blk = np.arange((m_now - 1) * b, m_now * b)
+            assert len(kept) == 4 and set(kept) <= set(blk)
+            logits = K[blk] @ Qd[pos]
+            want = sorted(blk[np.argsort(-logits, kind="stable")[:4]])   # single head: order of raw logits
+            assert list(kept) == want
+            n_glob += 4
+        assert len(cache.glob) == n_glob
+    assert n_glob == len(r["S"]) + 4 * ((L0 + steps - w) // b - r["m"])
+
+
+def test_decode_block_score_is_group_mean_of_block_softmaxes():
+    rng = _rng(14)
+    b, w, d, G = 4, 4, 6, 3
+    K = rng.standard_normal((8, d)) * 2
+    q = rng.standard_normal((G, d)) * 2
+    cache = O.DecodeCache(b=b, w=w, t_keep=2, sm_scale=0.5, glob=[], tail=list(range(7)))
+    kept = cache.append(7, q, K)
+    score = np.mean([sp_softmax((K[:4] @ q[g]) * 0.5) for g in range(G)], axis=0)
+    want = sorted(np.argsort(-score, kind="stable")[:2])
+    assert list(kept) == want
+
+
+# ----------------------------------------------------------------------------- Eq. 3: candidates
+def test_candidate_grid_closed_forms(golden):
+    g = golden("candidate_grid.txt")
+    b, M = int(g["block"][0]), int(g["M"][0])
+    C = O.candidate_grid(b, M, sigma=1.0)
+    assert C.shape == (M, 8)
+    np.testing.assert_allclose(C.sum(1), 1.0, rtol=1e-13)
+    # mu^1 = 0: p_2/p_1 = exp(-1/2); mu^M = log2 b: p_{b/2}/p_b = exp(-1/2)
+    assert g["mu_first"][0] == 0.0 and g["mu_last"][0] == 7.0
+    assert C[0, 1] / C[0, 0] == pytest.approx(math.exp(-0.5), rel=1e-12)
+    assert C[-1, -2] / C[-1, -1] == pytest.approx(math.exp(-0.5), rel=1e-12)
+    # mu^2 = log2(140/13): log-ratio of neighbours is linear in mu
+    mu2 = math.log2(g["mu_second_arg"][0])
+    assert math.log(C[1, 4] / C[1, 3]) == pytest.approx(-((4 - mu2) ** 2 - (3 - mu2) ** 2) / 2, rel=1e-11)
+    # budgets grow monotonically from efficiency- to accuracy-oriented
+    mean_keep = C @ O.retain_counts(b)
+    assert np.all(np.diff(mean_keep) > 0)
