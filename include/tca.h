@@ -1,0 +1,221 @@
+/*
+ * tca.h -- C ABI of the B200-native hot path of TCA-Attention
+ * (Training-free Context-adaptive Attention): score -> select -> compact ->
+ * sparse attention (prefill, decode) -> append/compress while decoding.
+ *
+ * Conventions
+ *   - Every pointer is labelled HOST or DEVICE.  All device buffers (inputs, outputs,
+ *     cache, workspace) are allocated and freed by the caller; the library allocates no
+ *     device memory and keeps no global state.
+ *   - Tensors are row-major with the head dimension contiguous:
+ *       Q [batch, n_q_heads, L, head_dim]      K, V [batch, n_kv_heads, L, head_dim]
+ *     A "unit" is one (sequence, KV head) pair, u = seq * n_kv_heads + kv_head; the G =
+ *     n_q_heads / n_kv_heads query heads kv_head*G .. kv_head*G+G-1 share it.
+ *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*); no call
+ *     synchronises the host.  Outputs are valid once the stream has been synchronised.
+ *   - Return value: TCA_OK or a negative error.  Argument errors are detected on the
+ *     host before anything is launched and leave every output untouched.  Unsupported
+ *     shapes return TCA_ERR_UNSUPPORTED; nothing ever falls back to the CPU.
+ *   - Identical inputs give bit-identical outputs (fixed split counts, fixed reduction
+ *     order, no floating-point atomics).
+ *   - Token positions are 0-based.
+ */
+#ifndef TCA_H_
+#define TCA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  TCA_OK = 0,
+  TCA_ERR_INVALID_ARG = -1, /* NULL / misaligned pointer, inconsistent sizes            */
+  TCA_ERR_UNSUPPORTED = -2, /* shape or dtype outside what the kernels implement        */
+  TCA_ERR_WORKSPACE = -3,   /* workspace smaller than tca_workspace_bytes() reports     */
+  TCA_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                   */
+  TCA_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (see tca_ws_status)   */
+  TCA_ERR_CAPACITY = -6     /* a cache region would overflow                            */
+};
+
+enum { TCA_F32 = 0, TCA_BF16 = 1 };
+
+/* tca_params.flags: run the prefill on the FP32 pipes even for bf16 inputs (the slow
+ * reference kernel the tensor-core kernel is cross-checked against). */
+enum { TCA_FLAG_PREFILL_SIMT = 1 };
+
+enum {
+  TCA_OP_SCORE = 0, TCA_OP_SELECT = 1, TCA_OP_COMPACT = 2,
+  TCA_OP_PREFILL = 3, TCA_OP_DECODE = 4, TCA_OP_APPEND = 5
+};
+
+/* Hyper-parameters of one attention layer (Algorithm 2, REQUIRE line). */
+typedef struct tca_params {
+  int32_t batch;      /* sequences                                                      */
+  int32_t n_q_heads;  /* multiple of n_kv_heads, group size G <= 8                      */
+  int32_t n_kv_heads;
+  int32_t head_dim;   /* d_h: 64 or 128                                                 */
+  int32_t block;      /* b: power of two, 1..128 (Section 4.1)                          */
+  int32_t window;     /* w >= 0: local subset size (Section 4)                          */
+  float alpha;        /* balance of Eq. 6, in [0, 1]                                    */
+  float sm_scale;     /* 1/sqrt(d_h) of Eqs. 2 and 5                                    */
+  int32_t dtype;      /* TCA_F32 or TCA_BF16: element type of Q, K, V, O and the cache  */
+  int32_t flags;      /* 0, or TCA_FLAG_* bits                                          */
+} tca_params;
+
+/* Number of int64 words per unit in tca_cache_desc.state. */
+#define TCA_STATE_WORDS 8
+enum {
+  TCA_ST_SEG_START = 0,  /* first cache row of the unit's segment                       */
+  TCA_ST_GLOBAL_CAP = 1, /* rows reserved for the global subset                         */
+  TCA_ST_N_GLOBAL = 2,   /* rows of the global subset in use                            */
+  TCA_ST_TAIL_HEAD = 3,  /* ring slot of the oldest tail token                          */
+  TCA_ST_N_TAIL = 4,     /* tokens in the tail ring                                     */
+  TCA_ST_SEQ_LEN = 5,    /* tokens seen so far = position of the next token             */
+  TCA_ST_T_KEEP = 6,     /* tokens kept from a block compressed while decoding          */
+  TCA_ST_RESERVED = 7
+};
+
+/*
+ * The retained KV cache ([K^G; K^L] of Eq. 2 kept across decode steps, Section 4.2 last
+ * paragraph).  All heads live in one flattened buffer with per-unit segments (the
+ * variable-length multi-head layout of Appendix C).  A unit's segment is
+ *     [ global region: global_cap rows | tail ring: tail_cap rows ]
+ * The global region holds the selected tokens S in ascending position; the ring holds
+ * the always-kept recent tokens, oldest at slot tail_head.
+ *
+ * The struct and its host arrays are owned by the caller and live in HOST memory; the
+ * k/v/pos/state buffers are DEVICE memory.  The host arrays mirror the device state
+ * words; lengths depend only on L, the number of appended tokens and the budget table,
+ * never on data, so both sides advance in lock step and no call reads the device back.
+ */
+typedef struct tca_cache_desc {
+  void* k;              /* DEVICE [rows_total, head_dim]                                */
+  void* v;              /* DEVICE [rows_total, head_dim]                                */
+  int32_t* pos;         /* DEVICE [rows_total]: original position of every row          */
+  int64_t* state;       /* DEVICE [n_units * TCA_STATE_WORDS]                           */
+  int64_t rows_total;
+  int64_t n_units;      /* batch * n_kv_heads                                           */
+  int64_t tail_cap;     /* ring capacity per unit; >= window + block for decoding       */
+  int64_t* seg_start;   /* HOST [n_units]  set by the caller                            */
+  int64_t* global_cap;  /* HOST [n_units]  set by the caller                            */
+  int64_t* n_global;    /* HOST [n_units]  maintained by the library                    */
+  int64_t* tail_head;   /* HOST [n_units]  maintained by the library                    */
+  int64_t* n_tail;      /* HOST [n_units]  maintained by the library                    */
+  int64_t* seq_len;     /* HOST [n_units]  maintained by the library                    */
+  int64_t* t_keep;      /* HOST [n_units]  set by the caller (tbar of tca_budget_resolve)*/
+} tca_cache_desc;
+
+const char* tca_strerror(int status);
+int tca_version(void);
+
+/*
+ * Budget map of Eq. 7 (Section 4.2), resolved on the host.
+ *   p       HOST [n_kv_heads, nK] double: configuration over K = {1, 2, 4, ..., 2^(nK-1)};
+ *           every row must be non-negative and sum to 1 within 1e-9.
+ *   m       number of blocks, m = max(0, floor((L - window) / block)).
+ *   n_k     HOST out [n_kv_heads, nK]: blocks that get retain count k.  floor(m * p_k) as
+ *           in Eq. 7, then the shortfall m - sum_k floor(m p_k) is handed out one each to
+ *           the largest fractional parts (ties to the larger k), so that Psi has exactly
+ *           m entries.
+ *   n_sel   HOST out [n_kv_heads]: size of the global subset, sum_k k * n_k.
+ *   tbar    HOST out [n_kv_heads]: floor(sum_k k * p_k), the decode-time retain count.
+ */
+int tca_budget_resolve(const double* p, int32_t n_kv_heads, int32_t nK, int64_t m,
+                       int32_t* n_k, int64_t* n_sel, int32_t* tbar);
+
+/* Bytes of DEVICE workspace `op` needs for sequence length L (for TCA_OP_DECODE and
+ * TCA_OP_APPEND, L is the total number of cache rows).  0 for an invalid request. */
+size_t tca_workspace_bytes(const tca_params* prm, int64_t L, int op);
+
+/*
+ * Token importance, Eq. 5 / Algorithm 2 line 1:  s = softmax(q_L K^T * sm_scale) over all
+ * L keys, per query head; the G distributions of a KV head's group are averaged.
+ *   q_last    DEVICE [batch, n_q_heads, head_dim]   query of the last token
+ *   K         DEVICE [batch, n_kv_heads, L, head_dim]
+ *   logscore  DEVICE out [batch, n_kv_heads, L] double: log s (s itself underflows at
+ *             long L).  Dot products are accumulated in fp64.
+ *   ws        DEVICE workspace, tca_workspace_bytes(prm, L, TCA_OP_SCORE), 256-B aligned
+ */
+int tca_score(const tca_params* prm, const void* q_last, const void* K, int64_t L,
+              double* logscore, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Core-context selection, Eqs. 6-8 / Algorithm 2 lines 2-6, one selection per unit.
+ * Blocks j < m of b tokens; h_j by Eq. 6; blocks ranked ascending by (h_j, j);
+ * t_j = Psi[rank_j]; the t_j tokens of block j with the largest score are kept, ties to
+ * the lower position.
+ *   logscore     DEVICE [batch, n_kv_heads, L] double
+ *   n_k          HOST [n_kv_heads, nK] from tca_budget_resolve (shared across the batch)
+ *   idx          DEVICE out int32, flattened: unit u owns idx[offsets[u] .. offsets[u+1]),
+ *                positions ascending
+ *   offsets_dev  DEVICE [n_units + 1] int64: exclusive prefix of n_sel over units
+ *   h_out        DEVICE out, optional (NULL to skip) [n_units, m] double
+ *   t_out        DEVICE out, optional (NULL to skip) [n_units, m] int32
+ */
+int tca_select(const tca_params* prm, const double* logscore, int64_t L,
+               const int32_t* n_k, int32_t nK, int32_t* idx, const int64_t* offsets_dev,
+               double* h_out, int32_t* t_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Upload the host mirror of `cache` (seg_start, global_cap, n_global, tail_head, n_tail,
+ * seq_len, t_keep) into cache->state.  Call once after filling the descriptor. */
+int tca_cache_init(const tca_params* prm, tca_cache_desc* cache, void* stream);
+
+/*
+ * Gather [K^G; K^L] (Eq. 2; "parallel tokens gathering", Appendix C): copy the rows of
+ * the selected set S into each unit's global region and the always-kept tail [m*b, L)
+ * into its ring, with their positions.  Sets n_global = n_sel, n_tail = L - m*b,
+ * tail_head = 0, seq_len = L on both the host mirror and the device state.
+ *   idx, offsets_dev  as written by / given to tca_select
+ *   offsets_host      HOST [n_units + 1] copy of offsets_dev
+ * TCA_ERR_CAPACITY if a unit's selection exceeds global_cap or its tail exceeds tail_cap.
+ */
+int tca_compact_kv(const tca_params* prm, const void* K, const void* V, int64_t L,
+                   const int32_t* idx, const int64_t* offsets_dev, const int64_t* offsets_host,
+                   tca_cache_desc* cache, void* stream);
+
+/*
+ * Sparse causal attention of the prefill, Eq. 2 / Algorithm 2 line 7.  Query i of a head
+ * attends to {j <= i : j in S or j >= c_i}, c_i = min(max(0, i - w + 1), m*b): its own
+ * last w keys (read from K, V) plus the selected keys before them (read from the cache's
+ * global region); every key is counted once.  O has the shape of Q.
+ *   ws   DEVICE workspace, tca_workspace_bytes(prm, L, TCA_OP_PREFILL); word 0 is a status
+ *        word readable with tca_ws_status.
+ */
+int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const void* V,
+                     int64_t L, const tca_cache_desc* cache, void* O,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * One decode step, Eq. 2 with a single query per head over the whole retained cache
+ * (global region + tail ring) of its KV head.
+ *   q  DEVICE [batch, n_q_heads, head_dim]     O  DEVICE out, same shape
+ *   ws DEVICE workspace, tca_workspace_bytes(prm, cache->rows_total, TCA_OP_DECODE)
+ */
+int tca_attn_decode(const tca_params* prm, const void* q, const tca_cache_desc* cache,
+                    void* O, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Append one token per sequence and compress when a block leaves the window (Section 4.2,
+ * "Online Token Selection in Decoding Stage").  The token goes to the tail ring; if the
+ * ring then holds window + block tokens, its oldest `block` tokens are scored with the
+ * current query (Eq. 5 restricted to the block, averaged over the query group), the top
+ * t_keep move to the end of the global region in ascending position and the rest are
+ * dropped.  Call before tca_attn_decode of the same step.
+ *   k_new, v_new  DEVICE [batch, n_kv_heads, head_dim]
+ *   q_cur         DEVICE [batch, n_q_heads, head_dim]  query of the appended token
+ * TCA_ERR_CAPACITY if the global region of a unit would overflow.
+ */
+int tca_cache_append(const tca_params* prm, tca_cache_desc* cache, const void* k_new,
+                     const void* v_new, const void* q_cur, void* stream);
+
+/* Synchronise `stream` and read the status word a kernel left at the start of a
+ * workspace: TCA_OK, or TCA_ERR_TIMEOUT if a bounded wait inside the kernel expired. */
+int tca_ws_status(const void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TCA_H_ */

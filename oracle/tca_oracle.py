@@ -143,8 +143,10 @@ def budget_map(n: Sequence[int], b: int) -> np.ndarray:
 
 def mean_retain_floor(p: Sequence[float], b: int) -> int:
     """t = floor(sum_k k * p_k): tokens kept from a block completed while decoding."""
-    return int(math.floor(float(np.dot(retain_counts(b).astype(np.float64),
-                                       np.asarray(p, dtype=np.float64)))))
+    total = 0.0
+    for k, pk in zip(retain_counts(b), np.asarray(p, dtype=np.float64)):
+        total += float(k) * float(pk)            # ascending k; k * p_k is exact (k = 2^i)
+    return int(math.floor(total))
 
 
 def rank_blocks(h: np.ndarray) -> np.ndarray:

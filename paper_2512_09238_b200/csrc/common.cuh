@@ -1,0 +1,172 @@
+// Shared declarations of the TCA-Attention kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tca.h"
+
+namespace tca {
+
+constexpr int kMaxGroup = 8;    // query heads per KV head
+constexpr int kMaxBlock = 128;  // b
+
+// ------------------------------------------------------------------ host-side checks
+#define TCA_CHECK_ARG(cond) \
+  do {                      \
+    if (!(cond)) return TCA_ERR_INVALID_ARG; \
+  } while (0)
+
+#define TCA_CHECK_CUDA(expr)                      \
+  do {                                            \
+    cudaError_t _e = (expr);                      \
+    if (_e != cudaSuccess) return TCA_ERR_CUDA;   \
+  } while (0)
+
+inline int check_launch() { return cudaGetLastError() == cudaSuccess ? TCA_OK : TCA_ERR_CUDA; }
+
+inline bool is_pow2(int64_t x) { return x > 0 && (x & (x - 1)) == 0; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Validates the hyper-parameters every entry point shares.
+int check_params(const tca_params* prm);
+
+inline int64_t num_blocks(const tca_params* prm, int64_t L) {
+  return L > prm->window ? (L - prm->window) / prm->block : 0;
+}
+inline int num_counts(const tca_params* prm) {  // |{1, 2, 4, ..., b}|
+  int n = 0;
+  for (int b = prm->block; b; b >>= 1) ++n;
+  return n;
+}
+inline size_t elt_size(int dtype) { return dtype == TCA_BF16 ? 2 : 4; }
+
+// ------------------------------------------------------------------ workspace layouts
+// score: logits [U][G][L] double, then partials [U][n_chunks][G][2] double.
+constexpr int kScoreChunkRows = 1024;  // rows of K per CTA of the logit kernel
+struct ScoreWs {
+  double* logits;
+  double* partials;
+  int64_t n_chunks;
+  size_t bytes;
+};
+ScoreWs score_ws_layout(const tca_params* prm, int64_t L, void* ws);
+
+// select: hkey [U][m] uint64, t [U][m] int32.
+struct SelectWs {
+  unsigned long long* hkey;
+  int32_t* t;
+  size_t bytes;
+};
+SelectWs select_ws_layout(const tca_params* prm, int64_t L, void* ws);
+
+// decode: partial (m, l, acc[d]) per (chunk, query head of the group).
+constexpr int kDecodeChunkRows = 256;  // cache rows per CTA of the split-KV kernel
+struct DecodeWs {
+  float* partial;     // [n_chunks_max][G][d + 2]
+  int64_t n_chunks_max;
+  size_t bytes;
+};
+DecodeWs decode_ws_layout(const tca_params* prm, int64_t rows_total, int64_t n_units, void* ws);
+
+// ------------------------------------------------------------------ device helpers
+#ifdef __CUDACC__
+
+template <typename T>
+struct Elt;
+template <>
+struct Elt<float> {
+  static constexpr int kDtype = TCA_F32;
+};
+template <>
+struct Elt<__nv_bfloat16> {
+  static constexpr int kDtype = TCA_BF16;
+};
+
+// Order-preserving map double -> uint64 (a < b  <=>  key(a) < key(b); -0 < +0).
+__device__ __forceinline__ unsigned long long ordered_key(double x) {
+  unsigned long long u = static_cast<unsigned long long>(__double_as_longlong(x));
+  return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
+}
+
+// bf16 bits -> double by bit placement (exact; subnormal bf16 inputs flush to zero,
+// which changes a dot product by less than 1e-36).
+__device__ __forceinline__ double bf16_bits_to_double(uint32_t bits16) {
+  uint32_t mag = bits16 & 0x7FFFu;
+  uint32_t hi = ((bits16 & 0x8000u) << 16) | ((mag << 13) + (896u << 20));
+  if ((mag >> 7) == 0) hi = (bits16 & 0x8000u) << 16;
+  return __hiloint2double(static_cast<int>(hi), 0);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t packed) { return __uint_as_float(packed & 0xFFFF0000u); }
+
+__device__ __forceinline__ double shfl_xor_double(double v, int mask) {
+  int lo = __double2loint(v), hi = __double2hiint(v);
+  lo = __shfl_xor_sync(0xffffffffu, lo, mask);
+  hi = __shfl_xor_sync(0xffffffffu, hi, mask);
+  return __hiloint2double(hi, lo);
+}
+__device__ __forceinline__ double shfl_double(double v, int src) {
+  int lo = __double2loint(v), hi = __double2hiint(v);
+  lo = __shfl_sync(0xffffffffu, lo, src);
+  hi = __shfl_sync(0xffffffffu, hi, src);
+  return __hiloint2double(hi, lo);
+}
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long v, int mask) {
+  return static_cast<unsigned long long>(
+      __double_as_longlong(shfl_xor_double(__longlong_as_double(static_cast<long long>(v)), mask)));
+}
+
+// Top-t of up to 128 keys held 4 per lane by one warp: MSB-first radix select on the
+// order-preserving 64-bit keys (radix 2, histogram = warp ballots), then ties at the
+// threshold go to the lowest token index.  Token i lives in lane i % 32, slot i / 32.
+// Returns per-slot keep flags as a 4-bit mask; `n_valid` tokens exist, t <= n_valid.
+__device__ __forceinline__ unsigned radix_select_top_t(const unsigned long long (&key)[4], int n_valid,
+                                                       int t, int lane) {
+  unsigned alive = 0;
+#pragma unroll
+  for (int s = 0; s < 4; ++s)
+    if (s * 32 + lane < n_valid) alive |= 1u << s;
+  unsigned keep = 0;
+  int need = t;
+  // Invariant: `need` more tokens must come from the alive set; all alive keys share the
+  // bits above the current one.
+  for (int bit = 63; bit >= 0 && need > 0; --bit) {
+    unsigned ones = 0;
+    int n_ones = 0, n_alive = 0;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      bool a = (alive >> s) & 1u;
+      bool one = a && ((key[s] >> bit) & 1ull);
+      if (one) ones |= 1u << s;
+      n_ones += __popc(__ballot_sync(0xffffffffu, one));
+      n_alive += __popc(__ballot_sync(0xffffffffu, a));
+    }
+    if (n_alive <= need) break;  // everything alive is kept
+    if (n_ones >= need) {
+      alive = ones;              // the threshold has this bit set; zeros are out
+    } else {
+      keep |= ones;              // all ones are above the threshold
+      need -= n_ones;
+      alive &= ~ones;
+    }
+  }
+  // Whatever is still alive is either all kept (n_alive <= need) or a set of equal keys
+  // of which the `need` lowest indices are kept.
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    bool a = (alive >> s) & 1u;
+    unsigned bal = __ballot_sync(0xffffffffu, a);
+    int before = __popc(bal & ((1u << lane) - 1u));
+    if (a && before < need) keep |= 1u << s;
+    need -= min(need, __popc(bal));
+  }
+  return keep;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace tca

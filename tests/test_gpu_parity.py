@@ -1,0 +1,283 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on
+seeded inputs small enough for the oracle yet spanning several tiles and ragged tails."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tca_oracle as O
+from paper_2512_09238_b200 import binding as B
+from paper_2512_09238_b200 import inputs as I
+import tca_harness as H
+
+pytestmark = pytest.mark.gpu
+
+BASE = I.WORKLOADS["config1"]
+SMALL = {
+    # the first benchmark configuration itself (fp32, 8 heads, L = 2048, b = 32, w = 128)
+    "config1": BASE,
+    # GQA 4:1, bf16, d = 128, ragged everywhere: L not a multiple of any tile, (L - w) % b != 0
+    "bf16_gqa4": BASE.scaled(name="bf16_gqa4", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, L=1500,
+                             dtype="bf16", block=64, window=256, seed=11, budget=("beta", 2.0, 5.0, 0.05, 1.0)),
+    "bf16_d64_g2": BASE.scaled(name="bf16_d64_g2", batch=1, n_q_heads=4, n_kv_heads=2, head_dim=64, L=777,
+                               dtype="bf16", block=16, window=100, seed=12),
+    "f32_d128_g8": BASE.scaled(name="f32_d128_g8", batch=1, n_q_heads=8, n_kv_heads=1, head_dim=128, L=600,
+                               dtype="f32", block=8, window=50, seed=13),
+    # 28/4 heads like Qwen2.5-7B: group of 7
+    "bf16_g7": BASE.scaled(name="bf16_g7", batch=1, n_q_heads=7, n_kv_heads=1, head_dim=128, L=1000,
+                           dtype="bf16", block=128, window=300, seed=14, budget=("fixed", 0.3)),
+    "f32_g3_b1": BASE.scaled(name="f32_g3_b1", batch=1, n_q_heads=3, n_kv_heads=1, head_dim=64, L=300,
+                             dtype="f32", block=1, window=17, seed=15, budget=("fixed", 1.0)),
+}
+
+
+@pytest.fixture(scope="module")
+def runs():
+    cache = {}
+
+    def get(name):
+        if name not in cache:
+            wl = SMALL[name]
+            data = I.generate(wl)
+            p = I.budget_table(wl)
+            run = H.gpu_select_compact(wl, data, p)
+            oracle = [[H.oracle_select_unit(wl, data, p, s, h, wl.L) for h in range(wl.n_kv_heads)]
+                      for s in range(wl.batch)]
+            cache[name] = (wl, data, p, run, oracle)
+        return cache[name]
+
+    return get
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_score_matches_oracle(runs, name):
+    wl, data, p, run, oracle = runs(name)
+    got = run.logscore.cpu().numpy()
+    for s in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            want = oracle[s][h]["log_s"]
+            u = s * wl.n_kv_heads + h
+            assert np.max(np.abs(got[u] - want)) < H.LOGSCORE_TOL
+            assert abs(np.exp(got[u]).sum() - 1) < 1e-6
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_selection_matches_oracle(runs, name):
+    wl, data, p, run, oracle = runs(name)
+    idx = run.idx.cpu().numpy()
+    t = run.t.cpu().numpy()
+    hh = run.h.cpu().numpy()
+    accepted = 0
+    for s in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            u = s * wl.n_kv_heads + h
+            res = oracle[s][h]
+            np.testing.assert_array_equal(run.n_k[h], res["n"])
+            S = idx[run.offsets[u]:run.offsets[u + 1]].astype(np.int64)
+            if res["m"]:
+                np.testing.assert_allclose(hh[u, :res["m"]], res["h"], rtol=2e-6, atol=1e-12)
+            accepted += H.compare_selection(res, S, t[u, :res["m"]], wl.block)
+    assert accepted <= 2, "differences inside the 1e-5 band should be rare"
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_compaction_is_bit_exact(runs, name):
+    wl, data, p, run, oracle = runs(name)
+    idx = run.idx.cpu().numpy()
+    Kc = run.cache.k.view(torch.int16 if wl.dtype == "bf16" else torch.int32).cpu().numpy()
+    Vc = run.cache.v.view(torch.int16 if wl.dtype == "bf16" else torch.int32).cpu().numpy()
+    pos = run.cache.pos.cpu().numpy()
+    state = run.cache.state.cpu().numpy().reshape(-1, B.TCA_STATE_WORDS)
+    raw = np.int16 if wl.dtype == "bf16" else np.int32
+    for s in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            u = s * wl.n_kv_heads + h
+            S = idx[run.offsets[u]:run.offsets[u + 1]].astype(np.int64)
+            T = O.retained_set(S, run.m, wl.block, wl.L)
+            rows = run.cache.unit_rows(u)
+            assert len(rows) == len(T)
+            np.testing.assert_array_equal(pos[rows], T)
+            np.testing.assert_array_equal(Kc[rows], data["k"][s, h, T].view(raw))
+            np.testing.assert_array_equal(Vc[rows], data["v"][s, h, T].view(raw))
+            assert state[u, 2] == len(S) and state[u, 4] == wl.L - run.m * wl.block and state[u, 5] == wl.L
+
+
+def _oracle_T(run, wl, u):
+    idx = run.idx.cpu().numpy()
+    S = idx[run.offsets[u]:run.offsets[u + 1]].astype(np.int64)
+    return O.retained_set(S, run.m, wl.block, wl.L)
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_prefill_matches_oracle_on_every_row(runs, name):
+    wl, data, p, run, oracle = runs(name)
+    out = H.from_device(H.gpu_prefill(run))
+    scale = H.scale_of(wl)
+    G = wl.group
+    for s in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            u = s * wl.n_kv_heads + h
+            T = _oracle_T(run, wl, u)                     # the GPU's own index set (see the 1e-5 rule)
+            K = I.widen(data["k"][s, h, :wl.L])
+            V = I.widen(data["v"][s, h, :wl.L])
+            for g in range(G):
+                Q = I.widen(data["q"][s, h * G + g, :wl.L])
+                want = O.attention_rows(Q, K, V, T, wl.window, scale)
+                H.check_attention(out[s, h * G + g], want, wl.dtype, f"{name} seq {s} head {h * G + g}")
+
+
+@pytest.mark.parametrize("name", ["bf16_gqa4", "bf16_d64_g2", "bf16_g7"])
+def test_bf16_prefill_reference_kernel_agrees(runs, name):
+    """The FP32-pipe kernel and the default bf16 kernel see the same inputs."""
+    wl, data, p, run, oracle = runs(name)
+    fast = H.from_device(H.gpu_prefill(run))
+    run.prm.flags = B.TCA_FLAG_PREFILL_SIMT
+    try:
+        slow = H.from_device(H.gpu_prefill(run))
+    finally:
+        run.prm.flags = 0
+    H.check_attention(fast, slow, "bf16", name)
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_decode_over_retained_cache(runs, name):
+    wl, data, p, run, oracle = runs(name)
+    L, G = wl.L, wl.group
+    q = run.dev["q"][:, :, L - 1, :].contiguous()
+    out = H.from_device(H.gpu_decode(run, q))
+    again = H.from_device(H.gpu_decode(run, q))
+    np.testing.assert_array_equal(out, again)            # fixed split and merge order
+    scale = H.scale_of(wl)
+    for s in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            T = _oracle_T(run, wl, s * wl.n_kv_heads + h)
+            K = I.widen(data["k"][s, h, :L])
+            V = I.widen(data["v"][s, h, :L])
+            for g in range(G):
+                qv = I.widen(data["q"][s, h * G + g, L - 1])
+                want = O.attention_over_set(qv, K[T], V[T], scale)
+                H.check_attention(out[s, h * G + g], want, wl.dtype, f"{name} decode")
+
+
+def test_hand_worked_selection_on_the_gpu(golden):
+    g = golden("hand_selection.txt")
+    b, w, L = int(g["block"][0]), int(g["window"][0]), int(g["length"][0])
+    prm = B.make_params(1, 1, 1, 64, b, w, alpha=g["alpha"][0], dtype=B.TCA_F32)
+    logscore = torch.from_numpy(np.log(np.array(g["s"]))).cuda().reshape(1, L)
+    n_k, n_sel, tbar = B.tca_budget_resolve(np.array([g["p"]]), int(g["m"][0]))
+    offsets = torch.tensor([0, int(n_sel[0])], dtype=torch.int64, device="cuda")
+    idx = torch.zeros(int(n_sel[0]), dtype=torch.int32, device="cuda")
+    h = torch.zeros(1, 5, dtype=torch.float64, device="cuda")
+    t = torch.zeros(1, 5, dtype=torch.int32, device="cuda")
+    B.tca_select(prm, logscore, L, n_k, idx, offsets, h, t, B.alloc_workspace(prm, L, B.TCA_OP_SELECT))
+    np.testing.assert_allclose(h.cpu().numpy()[0], g["h"], rtol=1e-6)
+    np.testing.assert_array_equal(t.cpu().numpy()[0], np.array(g["t"], dtype=int))
+    np.testing.assert_array_equal(idx.cpu().numpy(), np.array(g["S"], dtype=int))
+    assert tbar[0] == int(g["t_decode"][0])
+
+
+def test_full_budget_reproduces_dense_attention():
+    wl = SMALL["bf16_gqa4"].scaled(budget=("fixed", 1.0), seed=21, L=1100)
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    run = H.gpu_select_compact(wl, data, p)
+    assert int(run.n_sel.sum()) == wl.n_kv_heads * run.m * wl.block
+    out = H.from_device(H.gpu_prefill(run))
+    # independent dense reference: torch's causal attention in fp64 on the CPU
+    q = torch.from_numpy(I.widen(data["q"]))
+    k = torch.from_numpy(I.widen(data["k"])).repeat_interleave(wl.group, dim=1)
+    v = torch.from_numpy(I.widen(data["v"])).repeat_interleave(wl.group, dim=1)
+    att = (q @ k.transpose(-1, -2)) * H.scale_of(wl)
+    att = att.masked_fill(~torch.ones(wl.L, wl.L, dtype=torch.bool).tril(), float("-inf"))
+    want = (att.softmax(-1) @ v).numpy()
+    H.check_attention(out, want, "bf16", "dense special case")
+
+
+@pytest.mark.parametrize("L,w,b", [(100, 128, 32), (1, 4, 4), (64, 64, 16), (129, 1, 128)])
+def test_degenerate_lengths(L, w, b):
+    wl = BASE.scaled(batch=1, n_q_heads=2, n_kv_heads=2, head_dim=64, L=L, window=w, block=b, dtype="f32",
+                     seed=31, budget=("fixed", 0.5))
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    run = H.gpu_select_compact(wl, data, p)
+    out = H.from_device(H.gpu_prefill(run))
+    for h in range(2):
+        res = H.oracle_select_unit(wl, data, p, 0, h, L)
+        S = run.idx.cpu().numpy()[run.offsets[h]:run.offsets[h + 1]].astype(np.int64)
+        assert H.compare_selection(res, S, run.t.cpu().numpy()[h, :res["m"]], b) == 0
+        want = O.attention_rows(I.widen(data["q"][0, h]), I.widen(data["k"][0, h]), I.widen(data["v"][0, h]),
+                                res["T"], w, H.scale_of(wl))
+        H.check_attention(out[0, h], want, "f32", f"L={L}")
+
+
+@pytest.mark.parametrize("name,steps", [("bf16_gqa4", 150), ("bf16_d64_g2", 40), ("f32_g3_b1", 20),
+                                        ("f32_d128_g8", 30)])
+def test_append_compress_and_decode_steps(name, steps):
+    wl = SMALL[name].scaled(decode_steps=steps)
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    L, G, b, w = wl.L, wl.group, wl.block, wl.window
+    n_compress = (L + steps - w) // b - (L - w) // b
+    run = H.gpu_select_compact(wl, data, p, extra_blocks=n_compress + 1)
+    scale = H.scale_of(wl)
+    caches = {}
+    for s in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            u = s * wl.n_kv_heads + h
+            S = run.idx.cpu().numpy()[run.offsets[u]:run.offsets[u + 1]].astype(np.int64)
+            caches[u] = O.DecodeCache.from_prefill(S, run.m, L, b, w, p[h], scale)
+            assert caches[u].t_keep == run.tbar[h]
+    Kw, Vw, Qw = I.widen(data["k"]), I.widen(data["v"]), I.widen(data["q"])
+    dk, dv, dq = (H.to_device(data[x], wl.dtype) for x in ("k", "v", "q"))
+    fired = 0
+    for step in range(steps):
+        pos = L + step
+        B.tca_cache_append(run.prm, run.cache, dk[:, :, pos].contiguous(), dv[:, :, pos].contiguous(),
+                           dq[:, :, pos].contiguous())
+        out = H.from_device(H.gpu_decode(run, dq[:, :, pos].contiguous()))
+        cpos = run.cache.pos.cpu().numpy()
+        state = run.cache.state.cpu().numpy().reshape(-1, B.TCA_STATE_WORDS)
+        for s in range(wl.batch):
+            for h in range(wl.n_kv_heads):
+                u = s * wl.n_kv_heads + h
+                kept = caches[u].append(pos, Qw[s, h * G:(h + 1) * G, pos], Kw[s, h])
+                fired += kept is not None
+                rows = run.cache.unit_rows(u)
+                np.testing.assert_array_equal(cpos[rows], caches[u].positions())
+                assert state[u, 2] == run.cache.n_global[u] == len(caches[u].glob)
+                assert state[u, 4] == run.cache.n_tail[u] == len(caches[u].tail)
+                assert state[u, 3] == run.cache.tail_head[u] and state[u, 5] == pos + 1
+                if step % 7 == 0 or kept is not None or step == steps - 1:
+                    for g in range(G):
+                        want = caches[u].attend(Qw[s, h * G + g, pos], Kw[s, h], Vw[s, h])
+                        H.check_attention(out[s, h * G + g], want, wl.dtype, f"{name} step {step}")
+    assert fired == n_compress * wl.batch * wl.n_kv_heads and n_compress >= 1
+    # the compressed cache holds exactly the rows of K and V it claims to hold
+    raw = torch.int16 if wl.dtype == "bf16" else torch.int32
+    Kc = run.cache.k.view(raw).cpu().numpy()
+    for u, c in caches.items():
+        s, h = divmod(u, wl.n_kv_heads)
+        np.testing.assert_array_equal(Kc[run.cache.unit_rows(u)], data["k"][s, h, c.positions()].view(Kc.dtype))
+
+
+def test_capacity_and_workspace_errors():
+    wl = SMALL["bf16_d64_g2"]
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    run = H.gpu_select_compact(wl, data, p)
+    q = run.dev["q"][:, :, wl.L - 1, :].contiguous()
+    out = torch.empty_like(q)
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.TcaError) as e:
+        B.tca_attn_decode(run.prm, q, run.cache, out, small)
+    assert e.value.status == B.TCA_ERR_WORKSPACE
+    # a cache without room for the next compressed block refuses the append that would overflow it
+    steps_to_full = wl.window + wl.block - int(run.cache.n_tail[0])
+    k1, v1 = run.dev["k"][:, :, 0].contiguous(), run.dev["v"][:, :, 0].contiguous()
+    for _ in range(steps_to_full - 1):
+        B.tca_cache_append(run.prm, run.cache, k1, v1, q)
+    with pytest.raises(B.TcaError) as e:
+        B.tca_cache_append(run.prm, run.cache, k1, v1, q)
+    assert e.value.status == B.TCA_ERR_CAPACITY
+    torch.cuda.synchronize()
