@@ -1,0 +1,408 @@
+#!/usr/bin/env python
+"""Benchmark of the TCA-Attention hot path on B200 (one process per GPU).
+
+A step is one pass of the whole path over one batch of synthetic input: tca_score ->
+tca_select -> tca_compact_kv -> tca_attn_prefill at L tokens, then `decode_steps` x
+(tca_cache_append + tca_attn_decode).  Default workload: the 128K end-to-end
+configuration (one Llama-3-8B-shaped layer, 32/8 heads, d = 128, bf16, batch 1,
+L = 131072, 256 decode steps).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is prefill tokens/s over all GPUs with inputs
+resident in HBM; `decode_us_per_step` is the mean of the decode steps; `e2e` repeats the
+measurement through the same C-ABI calls with pinned HOST buffers copied in and the
+outputs copied back inside the timed region.  N > 1 runs N independent replicas (the
+path has no exchange step): no collective touches the data, only the timing is reduced.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+for _p in (ROOT, os.path.join(ROOT, "tests")):
+    if _p not in sys.path:
+        sys.path.insert(0, _p)
+
+METRIC = "128K prefill tok/s"
+UNIT = "tok/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [x for x in sm if x > 0]
+        return {"sm_mhz": float(np.median(busy)) if busy else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workload on the device
+class Pipeline:
+    def __init__(self, wl, data, p, torch, B, host_io: bool = False):
+        self.wl, self.torch, self.B = wl, torch, B
+        self.L, self.steps_decode = wl.L, wl.decode_steps
+        T = wl.L + wl.decode_steps
+        self.prm = B.make_params(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.block, wl.window,
+                                 alpha=wl.alpha, dtype=B.TCA_BF16 if wl.dtype == "bf16" else B.TCA_F32)
+        tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+
+        def host(a):
+            t = torch.from_numpy(a.view(np.int16) if wl.dtype == "bf16" else a)
+            return t.view(tdt) if wl.dtype == "bf16" else t
+
+        self.dev = {k: host(v).cuda() for k, v in data.items()}
+        U = wl.batch * wl.n_kv_heads
+        self.U = U
+        self.m = wl.n_blocks
+        self.n_k, self.n_sel, self.tbar = B.tca_budget_resolve(p, self.m)
+        per_unit = np.tile(self.n_sel, wl.batch)
+        self.offsets = np.zeros(U + 1, dtype=np.int64)
+        self.offsets[1:] = np.cumsum(per_unit)
+        self.offsets_dev = torch.from_numpy(self.offsets).cuda()
+        tk = np.tile(self.tbar, wl.batch).astype(np.int64)
+        n_compress = (wl.L + wl.decode_steps - wl.window) // wl.block - self.m
+        self.cache = B.Cache(self.prm, per_unit + (n_compress + 1) * tk, wl.window + wl.block, tk)
+        self.logscore = torch.empty(U, wl.L, dtype=torch.float64, device="cuda")
+        self.idx = torch.empty(max(1, int(self.offsets[-1])), dtype=torch.int32, device="cuda")
+        self.ws_score = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_SCORE)
+        self.ws_select = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_SELECT)
+        self.ws_prefill = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_PREFILL)
+        self.ws_decode = B.alloc_workspace(self.prm, self.cache.rows_total, B.TCA_OP_DECODE)
+        # device views used by the step (Q/K/V of the prompt are the first L tokens)
+        self.Qp = self.dev["q"][:, :, :wl.L].contiguous()
+        self.Kp = self.dev["k"][:, :, :wl.L].contiguous()
+        self.Vp = self.dev["v"][:, :, :wl.L].contiguous()
+        self.q_last = self.Qp[:, :, wl.L - 1].contiguous()
+        self.O = torch.empty_like(self.Qp)
+        # decode-step tensors laid out [step, B, H, d] so that a step is one contiguous slice
+        self.qd = self.dev["q"][:, :, wl.L:].permute(2, 0, 1, 3).contiguous()
+        self.kd = self.dev["k"][:, :, wl.L:].permute(2, 0, 1, 3).contiguous()
+        self.vd = self.dev["v"][:, :, wl.L:].permute(2, 0, 1, 3).contiguous()
+        self.Od = torch.empty_like(self.qd)
+        if host_io:
+            hq, hk, hv = host(data["q"]), host(data["k"]), host(data["v"])
+            self.h_Qp = hq[:, :, :wl.L].contiguous().pin_memory()
+            self.h_Kp = hk[:, :, :wl.L].contiguous().pin_memory()
+            self.h_Vp = hv[:, :, :wl.L].contiguous().pin_memory()
+            self.h_qd = hq[:, :, wl.L:].permute(2, 0, 1, 3).contiguous().pin_memory()
+            self.h_kd = hk[:, :, wl.L:].permute(2, 0, 1, 3).contiguous().pin_memory()
+            self.h_vd = hv[:, :, wl.L:].permute(2, 0, 1, 3).contiguous().pin_memory()
+            self.h_O = torch.empty_like(self.h_Qp).pin_memory()
+            self.h_Od = torch.empty_like(self.h_qd).pin_memory()
+        self.launches_per_step = 2 + 3 + 1 + 1 + wl.decode_steps * 3
+        self.ev = {}
+
+    def _ev(self, name):
+        e = self.torch.cuda.Event(enable_timing=True)
+        e.record()
+        self.ev.setdefault(name, []).append(e)
+
+    def step(self, host_io: bool = False, mark: bool = False):
+        B, prm, L = self.B, self.prm, self.L
+        if mark: self._ev("t_begin")
+        if host_io:
+            self.Qp.copy_(self.h_Qp, non_blocking=True)
+            self.Kp.copy_(self.h_Kp, non_blocking=True)
+            self.Vp.copy_(self.h_Vp, non_blocking=True)
+            self.q_last.copy_(self.Qp[:, :, L - 1])
+        if mark: self._ev("t0")
+        B.tca_score(prm, self.q_last, self.Kp, L, self.logscore, self.ws_score)
+        if mark: self._ev("t_score")
+        B.tca_select(prm, self.logscore, L, self.n_k, self.idx, self.offsets_dev, None, None, self.ws_select)
+        if mark: self._ev("t_select")
+        B.tca_compact_kv(prm, self.Kp, self.Vp, L, self.idx, self.offsets_dev, self.offsets, self.cache)
+        if mark: self._ev("t_compact")
+        B.tca_attn_prefill(prm, self.Qp, self.Kp, self.Vp, L, self.cache, self.O, self.ws_prefill)
+        if mark: self._ev("t_prefill")
+        if host_io:
+            self.h_O.copy_(self.O, non_blocking=True)
+            self.qd.copy_(self.h_qd, non_blocking=True)
+            self.kd.copy_(self.h_kd, non_blocking=True)
+            self.vd.copy_(self.h_vd, non_blocking=True)
+        if mark: self._ev("t_prefill_io")
+        for s in range(self.steps_decode):
+            B.tca_cache_append(prm, self.cache, self.kd[s], self.vd[s], self.qd[s])
+            B.tca_attn_decode(prm, self.qd[s], self.cache, self.Od[s], self.ws_decode)
+        if host_io:
+            self.h_Od.copy_(self.Od, non_blocking=True)
+        if mark: self._ev("t_decode")
+
+    def stage_ms(self):
+        """Mean milliseconds per stage over the marked steps."""
+        names = ["t_begin", "t0", "t_score", "t_select", "t_compact", "t_prefill", "t_prefill_io", "t_decode"]
+        out = {}
+        for a, b in zip(names[:-1], names[1:]):
+            out["h2d" if b == "t0" else b[2:]] = float(np.mean([x.elapsed_time(y) for x, y in zip(self.ev[a], self.ev[b])]))
+        return out
+
+    # ---- algorithmic work, counted from the realised index sets
+    def algorithmic_work(self):
+        wl = self.wl
+        idx = self.idx.cpu().numpy()
+        elt = 2 if wl.dtype == "bf16" else 4
+        d, L, w, G = wl.head_dim, wl.L, wl.window, wl.group
+        mb = self.m * wl.block
+        i = np.arange(L, dtype=np.int64)
+        c = np.minimum(np.maximum(0, i - w + 1), mb)
+        pairs = 0
+        for u in range(self.U):
+            S = idx[self.offsets[u]:self.offsets[u + 1]]
+            pairs += G * int((np.searchsorted(S, c, side="left") + (i - c + 1)).sum())
+        n_rows = (self.offsets[1:] - self.offsets[:-1]) + (L - mb)
+        dense_pairs = self.U * G * L * (L + 1) // 2
+        return {
+            "prefill_flops": 4.0 * d * pairs,
+            "dense_prefill_flops": 4.0 * d * dense_pairs,
+            "score_bytes": float(self.U * L * (d * elt + 8)),
+            "compact_bytes": float(2 * 2 * int(n_rows.sum()) * d * elt),
+            "decode_bytes_per_step": float(2 * int(n_rows.sum()) * d * elt),
+            "dense_decode_bytes_per_step": float(2 * self.U * L * d * elt),
+            "retained_fraction": float(n_rows.sum() / (self.U * L)),
+        }
+
+
+# ----------------------------------------------------------------------------- oracle timing (CPU baseline)
+def time_oracle(wl, data, p, budget_s: float = 20.0):
+    """The oracle as it stands on the host cores, on a bounded sample of the workload:
+    selection of ONE KV head at full length plus attention for a few query rows of one of
+    its query heads; the full prefill time is extrapolated from those two costs."""
+    from oracle import tca_oracle as O
+    import tca_harness as H
+    from paper_2512_09238_b200 import inputs as I
+    L, G = wl.L, wl.group
+    scale = H.scale_of(wl)
+    t0 = time.perf_counter()
+    K = I.widen(data["k"][0, 0, :L])
+    V = I.widen(data["v"][0, 0, :L])
+    res = O.select_head(I.widen(data["q"][0, :G, L - 1]), K, p[0], wl.block, wl.window, float(wl.alpha), scale)
+    t_select = time.perf_counter() - t0
+    Q = I.widen(data["q"][0, 0, :L])
+    rows = list(np.linspace(0, L - 1, 9).astype(int))
+    n_done, t1 = 0, time.perf_counter()
+    while n_done < 64 and (time.perf_counter() - t1) < max(2.0, budget_s - t_select):
+        O.attention_rows(Q, K, V, res["T"], wl.window, scale, rows=[rows[n_done % len(rows)]])
+        n_done += 1
+    t_row = (time.perf_counter() - t1) / max(1, n_done)
+    full = t_select * wl.batch * wl.n_kv_heads + t_row * L * wl.batch * wl.n_q_heads
+    return {"value": wl.batch * L / full, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "sample": f"select of 1 of {wl.batch * wl.n_kv_heads} KV heads at L={L} ({t_select:.2f} s) + "
+                      f"{n_done} query rows of 1 head ({t_row * 1e3:.1f} ms/row); prefill time extrapolated "
+                      f"to {wl.batch * wl.n_q_heads} heads x {L} rows"}
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="config4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--length", type=int, default=0, help="override L (smaller runs for profiling)")
+    ap.add_argument("--decode-steps", type=int, default=-1)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_2512_09238_b200 import inputs as I
+    wl = I.WORKLOADS[args.workload]
+    if args.length:
+        wl = wl.scaled(L=args.length)
+    if args.decode_steps >= 0:
+        wl = wl.scaled(decode_steps=args.decode_steps)
+    config = {"workload": f"{wl.name}: 1 attention layer, {wl.n_q_heads}/{wl.n_kv_heads} heads, d={wl.head_dim}, "
+                          f"{wl.dtype}, batch {wl.batch}, causal prefill L={wl.L} with selection and compaction, "
+                          f"then {wl.decode_steps} decode steps (append + attend)",
+              "block": wl.block, "window": wl.window, "alpha": wl.alpha, "seed": wl.seed,
+              "l2": "inputs larger than L2 (Q and O are 1 GiB each; a decode step streams the whole retained cache)",
+              "parallelism": "replicas only" if world > 1 else "1 GPU"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        data = I.generate(wl.scaled(seed=wl.seed))
+        p = I.budget_table(wl)
+        vals = []
+        for _ in range(args.warmup + args.steps):
+            vals.append(time_oracle(wl, data, p, budget_s=8.0))
+        vals = vals[args.warmup:]
+        v = float(np.mean([x["value"] for x in vals]))
+        base = dict(vals[-1])
+        base["value"] = v
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": wl.batch * wl.L / v * 1e3,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic", "config": config, "cpu_baseline": base,
+                          "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2512_09238_b200 import _build, binding as B
+    if rank == 0:
+        _build.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    B.lib()
+
+    wl_rank = wl.scaled(seed=wl.seed + 1000 * rank)        # every replica draws its own batch
+    data = I.generate(wl_rank)
+    p = I.budget_table(wl)
+    pipe = Pipeline(wl_rank, data, p, torch, B, host_io=not args.no_e2e)
+    peaks, peak_kind = load_peaks()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(host_io: bool):
+        pipe.ev = {}
+        for _ in range(args.warmup):
+            pipe.step(host_io=host_io)
+        barrier()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            pipe.step(host_io=host_io, mark=True)
+        e1.record()
+        barrier()
+        clocks = sampler.stop()
+        ms = e0.elapsed_time(e1)
+        stages = pipe.stage_ms()
+        if world > 1:
+            t = torch.tensor([ms] + [stages[k] for k in sorted(stages)], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t[0])
+            stages = {k: float(v) for k, v in zip(sorted(stages), t[1:])}
+        return ms / args.steps, stages, clocks
+
+    ms_step, stages, clocks = timed(host_io=False)
+    assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    work = pipe.algorithmic_work()
+    prefill_ms = stages["score"] + stages["select"] + stages["compact"] + stages["prefill"]
+    value = world * wl.batch * wl.L / (prefill_ms * 1e-3)
+    decode_us = stages["decode"] * 1e3 / max(1, wl.decode_steps)
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": config,
+           "decode_us_per_step": decode_us, "prefill_ms": prefill_ms, "clocks": clocks,
+           "gpu_launches": pipe.launches_per_step * args.steps}
+
+    tf_peak = peaks["bf16_tflops_sustained"]
+    achieved_tf = work["prefill_flops"] / (stages["prefill"] * 1e-3) / 1e12
+    out["roofline"] = {"kernel": "tca_attn_prefill", "bound": "tensor", "achieved": achieved_tf, "peak": tf_peak,
+                       "unit": "TFLOP/s", "frac": achieved_tf / tf_peak, "traffic": None,
+                       "peak_kind": f"bf16 sustained, {peak_kind}", "frac_of_burst": achieved_tf / peaks["bf16_tflops"]}
+    hbm = peaks["hbm_gbs"]
+
+    def hbm_stage(bytes_, ms):
+        gbs = bytes_ / (ms * 1e-3) / 1e9
+        return {"ms": ms, "bytes": bytes_, "achieved_gbs": gbs, "frac_of_measured": gbs / hbm, "frac_of_8tbs": gbs / 8000.0}
+
+    out["stages"] = {
+        "score": hbm_stage(work["score_bytes"], stages["score"]),
+        "select": {"ms": stages["select"]},
+        "compact": hbm_stage(work["compact_bytes"], stages["compact"]),
+        "prefill": {"ms": stages["prefill"], "flops": work["prefill_flops"], "dense_flops": work["dense_prefill_flops"]},
+        "decode_step": hbm_stage(work["decode_bytes_per_step"], decode_us * 1e-3),
+        "retained_fraction": work["retained_fraction"],
+        "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
+    }
+
+    if not args.no_e2e:
+        ms_e2e, st_e2e, _ = timed(host_io=True)
+        elt = 2 if wl.dtype == "bf16" else 4
+        nQ = wl.batch * wl.n_q_heads * wl.head_dim * elt
+        nKV = wl.batch * wl.n_kv_heads * wl.head_dim * elt
+        h2d = wl.L * (nQ + 2 * nKV) + wl.decode_steps * (nQ + 2 * nKV)
+        d2h = wl.L * nQ + wl.decode_steps * nQ
+        e2e_prefill_ms = sum(st_e2e[k] for k in ("h2d", "score", "select", "compact", "prefill", "prefill_io"))
+        out["e2e"] = {"value": world * wl.batch * wl.L / (e2e_prefill_ms * 1e-3), "unit": UNIT,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
+                      "prefill_ms": e2e_prefill_ms,
+                      "decode_us_per_step": st_e2e["decode"] * 1e3 / max(1, wl.decode_steps),
+                      "note": "same calls with pinned host buffers: Q, K, V copied in and O copied back inside "
+                              "the timed prefill; decode tokens copied in, decode outputs copied back"}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = time_oracle(wl_rank, data, p)
+
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
