@@ -37,7 +37,8 @@ enum {
   TCA_ERR_WORKSPACE = -3,   /* workspace smaller than tca_workspace_bytes() reports     */
   TCA_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                   */
   TCA_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (see tca_ws_status)   */
-  TCA_ERR_CAPACITY = -6     /* a cache region would overflow                            */
+  TCA_ERR_CAPACITY = -6,    /* a cache region would overflow                            */
+  TCA_ERR_SCRATCH_LIMIT = -7 /* problem larger than the built-in scratch of a *_static call */
 };
 
 enum { TCA_F32 = 0, TCA_BF16 = 1 };
@@ -210,6 +211,38 @@ int tca_attn_decode(const tca_params* prm, const void* q, const tca_cache_desc* 
  */
 int tca_cache_append(const tca_params* prm, tca_cache_desc* cache, const void* k_new,
                      const void* v_new, const void* q_cur, void* stream);
+
+/* Size of the scratch array built into the library image for tca_attn_decode_static. */
+#define TCA_DECODE_STATIC_SCRATCH_BYTES (16u << 20)
+
+/*
+ * tca_attn_decode for callers that must not allocate.  (The paper has no counterpart;
+ * this is a deployment convenience.)  Some hosts of this library cannot hand it a
+ * workspace: a plug-in inside a serving engine that has already claimed all device memory
+ * for its own pool, a latency-critical loop in which cudaMalloc's implicit device-wide
+ * synchronisation is not acceptable, or glue code that simply has no allocator at hand.
+ * This variant computes exactly what tca_attn_decode computes, with the split-KV partial
+ * results kept in a fixed TCA_DECODE_STATIC_SCRATCH_BYTES (16 MiB) array that is part of
+ * the library image: every GPU that loads the library holds those 16 MiB until the
+ * process exits, and the call performs no cudaMalloc, cudaFree or other allocation.
+ *
+ *   q, cache, O, stream   as for tca_attn_decode; inputs and outputs still belong to the
+ *                         caller.
+ *   Limit   the partials need (rows_total / 256 + 2 * n_units + 1) * G * (head_dim + 2) * 4
+ *           bytes; a cache for which that exceeds the array (about 2 million rows at
+ *           G = 4, head_dim = 128) is refused with TCA_ERR_SCRATCH_LIMIT and nothing is
+ *           launched.  Use tca_attn_decode with a workspace of your own for larger caches.
+ *   Set-up  the first call on each device looks up the array's device address (with that
+ *           device current) and remembers it; make that first call outside any stream
+ *           capture.
+ *   Sharing every call on a device uses the same array, which keeps the previous call's
+ *           contents.  Nothing in it has to start at zero (each partial is written before
+ *           it is read), but two calls that overlap on the GPU (different streams, or
+ *           different threads without ordering) race on it and corrupt each other:
+ *           serialise them.
+ */
+int tca_attn_decode_static(const tca_params* prm, const void* q, const tca_cache_desc* cache,
+                           void* O, void* stream);
 
 /* Synchronise `stream` and read the status word a kernel left at the start of a
  * workspace: TCA_OK, or TCA_ERR_TIMEOUT if a bounded wait inside the kernel expired. */

@@ -19,7 +19,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libtca.so")
 
 TCA_OK, TCA_ERR_INVALID_ARG, TCA_ERR_UNSUPPORTED, TCA_ERR_WORKSPACE = 0, -1, -2, -3
-TCA_ERR_CUDA, TCA_ERR_TIMEOUT, TCA_ERR_CAPACITY = -4, -5, -6
+TCA_ERR_CUDA, TCA_ERR_TIMEOUT, TCA_ERR_CAPACITY, TCA_ERR_SCRATCH_LIMIT = -4, -5, -6, -7
+TCA_DECODE_STATIC_SCRATCH_BYTES = 16 << 20
 TCA_F32, TCA_BF16 = 0, 1
 TCA_FLAG_PREFILL_SIMT = 1
 TCA_OP_SCORE, TCA_OP_SELECT, TCA_OP_COMPACT, TCA_OP_PREFILL, TCA_OP_DECODE, TCA_OP_APPEND = range(6)
@@ -28,7 +29,7 @@ TCA_STATE_WORDS = 8
 EXPORTS = (
     "tca_strerror", "tca_version", "tca_budget_resolve", "tca_workspace_bytes", "tca_score",
     "tca_select", "tca_cache_init", "tca_compact_kv", "tca_attn_prefill", "tca_attn_decode",
-    "tca_cache_append", "tca_ws_status",
+    "tca_cache_append", "tca_ws_status", "tca_attn_decode_static",
 )
 
 
@@ -82,6 +83,7 @@ def lib() -> C.CDLL:
         L.tca_attn_decode.argtypes = [P, vp, D, vp, vp, sz, vp]
         L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
         L.tca_ws_status.argtypes = [vp, vp]
+        L.tca_attn_decode_static.argtypes = [P, vp, D, vp, vp]
         for name in EXPORTS:
             if name not in ("tca_strerror", "tca_workspace_bytes"):
                 getattr(L, name).restype = C.c_int
@@ -189,6 +191,15 @@ def tca_attn_prefill(prm, Q, K, V, L, cache: "Cache", O, ws, stream=None) -> Non
 def tca_attn_decode(prm, q, cache: "Cache", O, ws, stream=None) -> None:
     _check(lib().tca_attn_decode(C.byref(prm), _dev(q), C.byref(cache.desc), _dev(O), *_ws_args(ws),
                                  _stream(stream)), "tca_attn_decode")
+
+
+def tca_attn_decode_static(prm, q, cache: "Cache", O, stream=None) -> None:
+    """tca_attn_decode without a workspace: the partials live in a 16 MiB array inside the
+    library, so the call allocates nothing.  For callers that cannot allocate device memory
+    (all of it owned by a host engine's pool, or no allocator available in a latency-critical
+    loop).  Calls share that array: do not let two of them overlap on the GPU."""
+    _check(lib().tca_attn_decode_static(C.byref(prm), _dev(q), C.byref(cache.desc), _dev(O), _stream(stream)),
+           "tca_attn_decode_static")
 
 
 def tca_cache_append(prm, cache: "Cache", k_new, v_new, q_cur, stream=None) -> None:

@@ -73,6 +73,7 @@ const char* tca_strerror(int status) {
     case TCA_ERR_CUDA: return "CUDA runtime error";
     case TCA_ERR_TIMEOUT: return "device-side wait timed out";
     case TCA_ERR_CAPACITY: return "cache capacity exceeded";
+    case TCA_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the static entry point";
     default: return "unknown status";
   }
 }

@@ -10,6 +10,8 @@
 //                         un-normalised partial (acc, max, sum) per (chunk, query head).
 //   decode_combine_kernel merges a unit's partials in chunk order (fixed order => bit-
 //                         reproducible) and normalises.
+#include <mutex>
+
 #include "common.cuh"
 #include "rowslice.cuh"
 
@@ -301,6 +303,72 @@ extern "C" int tca_attn_decode(const tca_params* prm, const void* q, const tca_c
   TCA_CHECK_ARG(c->n_units == U && U <= 65535);
   DecodeWs lay = decode_ws_layout(prm, c->rows_total, U, ws);
   if (ws_bytes < lay.bytes) return TCA_ERR_WORKSPACE;
+  int64_t max_len = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    const int64_t len = c->n_global[u] + c->n_tail[u];
+    max_len = len > max_len ? len : max_len;
+  }
+  TCA_CHECK_ARG(max_len >= 1);
+  const int G = prm->n_q_heads / prm->n_kv_heads;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (prm->dtype == TCA_BF16) {
+    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, s);
+    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, s);
+  }
+  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, s);
+  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, s);
+}
+
+// ---------------------------------------------------------------------------------------
+// Decode without any allocation: the split-KV partials live in a fixed array inside the
+// library image instead of a caller-provided workspace.
+namespace tca {
+namespace {
+
+constexpr size_t kStaticScratchBytes = size_t(TCA_DECODE_STATIC_SCRATCH_BYTES);
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
+
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of g_decode_scratch on the current device.  In host code the array's
+// name is only a handle; the address a kernel can use comes from cudaGetSymbolAddress,
+// looked up once per device with that device current.
+int static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TCA_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return TCA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (g_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_decode_scratch) != cudaSuccess || p == nullptr) return TCA_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  *out = g_scratch_addr[dev];
+  return TCA_OK;
+}
+
+}  // namespace
+}  // namespace tca
+
+extern "C" int tca_attn_decode_static(const tca_params* prm, const void* q, const tca_cache_desc* c, void* O,
+                                      void* stream) {
+  int st = check_params(prm);
+  if (st != TCA_OK) return st;
+  TCA_CHECK_ARG(q && c && O);
+  TCA_CHECK_ARG(c->k && c->v && c->state && c->n_global && c->n_tail);
+  TCA_CHECK_ARG(aligned(q, 16) && aligned(O, 16) && aligned(c->k, 16) && aligned(c->v, 16));
+  const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
+  TCA_CHECK_ARG(c->n_units == U && U <= 65535);
+  // same layout as the workspace variant; refuse what does not fit the built-in array
+  DecodeWs lay = decode_ws_layout(prm, c->rows_total, U, nullptr);
+  if (lay.bytes > kStaticScratchBytes) return TCA_ERR_SCRATCH_LIMIT;
+  void* scratch = nullptr;
+  st = static_scratch(&scratch);
+  if (st != TCA_OK) return st;
+  lay = decode_ws_layout(prm, c->rows_total, U, scratch);
   int64_t max_len = 0;
   for (int64_t u = 0; u < U; ++u) {
     const int64_t len = c->n_global[u] + c->n_tail[u];
