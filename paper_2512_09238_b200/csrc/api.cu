@@ -8,6 +8,8 @@
 
 namespace tca {
 
+size_t prefill_tc_ws_bytes(const tca_params* prm);
+
 int check_params(const tca_params* prm) {
   TCA_CHECK_ARG(prm != nullptr);
   TCA_CHECK_ARG(prm->batch >= 1 && prm->n_kv_heads >= 1 && prm->n_q_heads >= 1);
@@ -131,7 +133,7 @@ size_t tca_workspace_bytes(const tca_params* prm, int64_t L, int op) {
     case TCA_OP_SCORE: return score_ws_layout(prm, L, nullptr).bytes;
     case TCA_OP_SELECT: return select_ws_layout(prm, L, nullptr).bytes;
     case TCA_OP_COMPACT: return 256;
-    case TCA_OP_PREFILL: return 4096;
+    case TCA_OP_PREFILL: return align_up(prefill_tc_ws_bytes(prm), 256);
     case TCA_OP_DECODE: return decode_ws_layout(prm, L, U, nullptr).bytes;
     case TCA_OP_APPEND: return 256;
     default: return 0;

@@ -7,6 +7,9 @@ namespace tca {
 template <typename T, int D>
 int launch_prefill_simt(const tca_params*, const void*, const void*, const void*, int64_t,
                         const tca_cache_desc*, void*, cudaStream_t);
+template <int D>
+int launch_prefill_tc(const tca_params*, const void*, const void*, const void*, int64_t, const tca_cache_desc*,
+                      void*, void*, cudaStream_t);
 }  // namespace tca
 
 using namespace tca;
@@ -31,6 +34,11 @@ extern "C" int tca_attn_prefill(const tca_params* prm, const void* Q, const void
     if (prm->head_dim == 128) return launch_prefill_simt<float, 128>(prm, Q, K, V, L, c, O, s);
     return launch_prefill_simt<float, 64>(prm, Q, K, V, L, c, O, s);
   }
-  if (prm->head_dim == 128) return launch_prefill_simt<__nv_bfloat16, 128>(prm, Q, K, V, L, c, O, s);
-  return launch_prefill_simt<__nv_bfloat16, 64>(prm, Q, K, V, L, c, O, s);
+  if (prm->flags & TCA_FLAG_PREFILL_SIMT) {
+    if (prm->head_dim == 128) return launch_prefill_simt<__nv_bfloat16, 128>(prm, Q, K, V, L, c, O, s);
+    return launch_prefill_simt<__nv_bfloat16, 64>(prm, Q, K, V, L, c, O, s);
+  }
+  TCA_CHECK_ARG(c->seg_start && c->n_global);
+  if (prm->head_dim == 128) return launch_prefill_tc<128>(prm, Q, K, V, L, c, O, ws, s);
+  return launch_prefill_tc<64>(prm, Q, K, V, L, c, O, ws, s);
 }

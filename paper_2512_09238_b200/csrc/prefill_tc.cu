@@ -1,0 +1,427 @@
+// Sparse causal prefill attention (Eq. 2, Algorithm 2 line 7) on the 5th-generation tensor
+// cores: tcgen05.mma with fp32 accumulators in TMEM, operands staged by TMA with 128-byte
+// swizzle, online softmax on the CUDA cores, bf16 inputs.
+//
+// One CTA owns 128 consecutive query positions of TWO query heads of one GQA group (same
+// KV head, same positions, hence the same key tiles and the same mask), which halves the
+// K/V traffic per flop and lets the tensor pipe work on one head while the other head's
+// softmax runs.  Key tiles (128 keys) come from two ranges under one online softmax:
+//   (1) the unit's selected keys in the cache's global region with position < c_hi, read
+//       through a per-unit tensor map whose bound is the region's length, and
+//   (2) the contiguous band [c_lo, i_last] of the original K/V,
+// with c_i = min(max(0, i - w + 1), m*b); row i sees columns {pos < c_i} of (1) and
+// {c_i <= j <= i} of (2), so every key is counted once.  Only tiles that straddle one of
+// those bounds evaluate a mask.
+//
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 /
+// 6-9 = softmax of head 0 / head 1 (one thread per query row = one TMEM lane).
+// TMEM (512 columns): S0 | S1 | O0 | O1.  Shared memory: Q0 Q1 | 3-slot K/V ring | P0 P1.
+// Per tile the issuer runs  PV0(t) S0(t+1) PV1(t) S1(t+1)  so that S of one head is being
+// computed while the other head's softmax is in flight.  O stays in TMEM and is rescaled
+// lazily: only when a row maximum grew by more than 2^8 since the last rescale.
+//
+// Every mbarrier wait is bounded; a wait that gives up raises the status word of the
+// workspace, lets outstanding copies land, frees TMEM and returns.
+#include <cuda.h>
+
+#include <vector>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace tca {
+namespace {
+
+constexpr int BM = 128, BN = 128;
+constexpr int kThreads = 320;
+constexpr int kRing = 3;
+constexpr int kHalfBytes = 128 * 128;  // 128 rows x 128 bytes (64 bf16): one swizzled box
+constexpr float kRescaleThreshold = 8.f;
+
+template <int D>
+struct TcCfg {
+  static constexpr int NH = D / 64;                 // 64-element halves per row
+  static constexpr int kQ = NH * kHalfBytes;        // one head's Q tile
+  static constexpr int kKV = NH * kHalfBytes;       // one K or V tile
+  static constexpr int kP = 2 * kHalfBytes;         // 128 x 128 bf16
+  static constexpr int offQ = 0;
+  static constexpr int offKV = 2 * kQ;
+  static constexpr int offP = offKV + kRing * kKV;
+  static constexpr int offBar = offP + 2 * kP;
+  static constexpr int bytes = offBar + 256 + 1024;  // + barriers/scalars + alignment slack
+  static constexpr uint32_t colS(int h) { return uint32_t(h) * 128u; }
+  static constexpr uint32_t colO(int h) { return 256u + uint32_t(h) * uint32_t(D); }
+};
+
+enum { BAR_Q = 0, BAR_FULL = 1, BAR_EMPTY = 4, BAR_S = 7, BAR_P = 9, BAR_PV = 11, N_BARS = 13 };
+
+struct TileGeom {
+  int n_gt, nt;
+  int64_t c_lo;
+  __device__ __forceinline__ bool is_global(int t) const { return t < n_gt; }
+  __device__ __forceinline__ int64_t first(int t) const {  // first cache row / first position
+    return t < n_gt ? int64_t(t) * BN : c_lo + int64_t(t - n_gt) * BN;
+  }
+};
+
+__device__ __forceinline__ int lower_bound_pos(const int32_t* pos, int n, int64_t bound) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (int64_t(pos[mid]) < bound) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restrict__ pos,
+                  const int64_t* __restrict__ state, int64_t L, int n_q_heads, int n_kv_heads, int window,
+                  int64_t mb, float scale_log2e, __nv_bfloat16* __restrict__ O, int* __restrict__ status,
+                  int n_qtiles, int pairs_per_unit) {
+  using Cfg = TcCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::offBar);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* s_nvis = reinterpret_cast<int*>(tmem_slot + 2);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = n_q_heads / n_kv_heads;
+  const int U = int(gridDim.x) / (n_qtiles * pairs_per_unit);
+  const int per_tile = U * pairs_per_unit;
+  const int tile = n_qtiles - 1 - int(blockIdx.x) / per_tile;   // long rows first
+  const int rem = int(blockIdx.x) % per_tile;
+  const int u = rem / pairs_per_unit, pair = rem % pairs_per_unit;
+  const int nh = min(2, G - 2 * pair);                          // heads handled here
+  const int seq = u / n_kv_heads, kvh = u % n_kv_heads;
+  const int hq0 = seq * n_q_heads + kvh * G + 2 * pair;         // first query head (flattened over batch)
+
+  const int64_t i0 = int64_t(tile) * BM;
+  const int64_t i_last = min(i0 + BM - 1, L - 1);
+  const int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
+  const int64_t seg = st[TCA_ST_SEG_START];
+  const int n_global = int(st[TCA_ST_N_GLOBAL]);
+  const int64_t c_lo = min(max(int64_t(0), i0 - window + 1), mb);
+  const int64_t c_hi = min(max(int64_t(0), i_last - window + 1), mb);
+
+  if (tid == 0) {
+    ptx::mbar_init(&bars[BAR_Q], 1);
+    for (int i = 0; i < kRing; ++i) { ptx::mbar_init(&bars[BAR_FULL + i], 1); ptx::mbar_init(&bars[BAR_EMPTY + i], 1); }
+    for (int h = 0; h < 2; ++h) {
+      ptx::mbar_init(&bars[BAR_S + h], 1);
+      ptx::mbar_init(&bars[BAR_P + h], 128);
+      ptx::mbar_init(&bars[BAR_PV + h], 1);
+    }
+    ptx::fence_barrier_init();
+    *abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
+    *s_nvis = lower_bound_pos(pos + seg, n_global, c_hi);
+  }
+  if (warp == 0) {
+    ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  TileGeom geo;
+  geo.n_gt = (*s_nvis + BN - 1) / BN;
+  geo.c_lo = c_lo;
+  geo.nt = geo.n_gt + int((i_last - c_lo + BN) / BN);
+  const int nt = geo.nt;
+
+  if (!*abort_flag) {
+    if (warp == 0) {
+      // ------------------------------------------------------------- TMA producer
+      if (lane == 0) {
+        ptx::mbar_arrive_expect_tx(&bars[BAR_Q], uint32_t(nh * Cfg::kQ));
+        for (int h = 0; h < nh; ++h)
+          for (int half = 0; half < Cfg::NH; ++half)
+            ptx::tma_load_3d(smem + Cfg::offQ + h * Cfg::kQ + half * kHalfBytes, &maps[0], half * 64, int(i0),
+                             hq0 + h, &bars[BAR_Q]);
+        for (int n = 0; n < 2 * nt; ++n) {
+          const int t = n >> 1, is_v = n & 1, slot = n % kRing;
+          if (n >= kRing && !ptx::mbar_wait(&bars[BAR_EMPTY + slot], uint32_t(n / kRing - 1) & 1u, abort_flag)) break;
+          ptx::mbar_arrive_expect_tx(&bars[BAR_FULL + slot], uint32_t(Cfg::kKV));
+          uint8_t* dst = smem + Cfg::offKV + slot * Cfg::kKV;
+          const int y = int(geo.first(t));
+          for (int half = 0; half < Cfg::NH; ++half) {
+            if (geo.is_global(t))
+              ptx::tma_load_2d(dst + half * kHalfBytes, &maps[3 + 2 * u + is_v], half * 64, y, &bars[BAR_FULL + slot]);
+            else
+              ptx::tma_load_3d(dst + half * kHalfBytes, &maps[1 + is_v], half * 64, y, u, &bars[BAR_FULL + slot]);
+          }
+        }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------- MMA issuer
+      if (lane == 0) {
+        constexpr uint32_t idescS = ptx::idesc_bf16(BM, BN, false);
+        constexpr uint32_t idescPV = ptx::idesc_bf16(BM, D, true);
+        const uint32_t q_base = ptx::smem_u32(smem + Cfg::offQ);
+        const uint32_t kv_base = ptx::smem_u32(smem + Cfg::offKV);
+        const uint32_t p_base = ptx::smem_u32(smem + Cfg::offP);
+        auto issue_S = [&](int h, int slot) {
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = uint32_t(kk >> 2) * kHalfBytes + uint32_t(kk & 3) * 32u;
+            const uint64_t a = ptx::smem_desc_sw128(q_base + h * Cfg::kQ + off, 16, 1024);
+            const uint64_t b = ptx::smem_desc_sw128(kv_base + slot * Cfg::kKV + off, 16, 1024);
+            ptx::umma_ss(tmem_base + Cfg::colS(h), a, b, idescS, kk > 0);
+          }
+        };
+        auto issue_PV = [&](int h, int slot, bool acc) {
+#pragma unroll
+          for (int kk = 0; kk < BN / 16; ++kk) {
+            const uint32_t offp = uint32_t(kk >> 2) * kHalfBytes + uint32_t(kk & 3) * 32u;
+            const uint64_t a = ptx::smem_desc_sw128(p_base + h * Cfg::kP + offp, 16, 1024);
+            const uint64_t b = ptx::smem_desc_sw128(kv_base + slot * Cfg::kKV + uint32_t(kk) * 2048u, kHalfBytes, 1024);
+            ptx::umma_ss(tmem_base + Cfg::colO(h), a, b, idescPV, (acc || kk > 0) ? 1u : 0u);
+          }
+        };
+        bool ok = ptx::mbar_wait(&bars[BAR_Q], 0, abort_flag) && ptx::mbar_wait(&bars[BAR_FULL + 0], 0, abort_flag);
+        if (ok) {
+          ptx::tc_fence_after();
+          for (int h = 0; h < nh; ++h) { issue_S(h, 0); ptx::umma_commit(&bars[BAR_S + h]); }
+          ptx::umma_commit(&bars[BAR_EMPTY + 0]);
+        }
+        for (int t = 0; t < nt && ok; ++t) {
+          const int nV = 2 * t + 1, slotV = nV % kRing;
+          const int nK = 2 * t + 2, slotK = nK % kRing;
+          ok = ptx::mbar_wait(&bars[BAR_FULL + slotV], uint32_t(nV / kRing) & 1u, abort_flag);
+          for (int h = 0; h < nh && ok; ++h) {
+            ok = ptx::mbar_wait(&bars[BAR_P + h], uint32_t(t) & 1u, abort_flag);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            issue_PV(h, slotV, t > 0);
+            ptx::umma_commit(&bars[BAR_PV + h]);
+            if (h == nh - 1) ptx::umma_commit(&bars[BAR_EMPTY + slotV]);
+            if (t + 1 < nt) {
+              if (h == 0) {
+                ok = ptx::mbar_wait(&bars[BAR_FULL + slotK], uint32_t(nK / kRing) & 1u, abort_flag);
+                if (!ok) break;
+                ptx::tc_fence_after();
+              }
+              issue_S(h, slotK);
+              ptx::umma_commit(&bars[BAR_S + h]);
+              if (h == nh - 1) ptx::umma_commit(&bars[BAR_EMPTY + slotK]);
+            }
+          }
+        }
+      }
+    } else {
+      // ------------------------------------------------------------- softmax, one row per thread
+      const int h = (warp - 2) >> 2;
+      if (h < nh) {
+        const int quarter = warp & 3;                    // TMEM lanes this warp may touch
+        const int row = quarter * 32 + lane;
+        const int64_t i = i0 + row;
+        const int64_t c_i = min(max(int64_t(0), i - window + 1), mb);
+        const int nvis_i = lower_bound_pos(pos + seg, n_global, c_i);
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
+        uint8_t* p_row = smem + Cfg::offP + h * Cfg::kP + row * 128;
+        float m_run = -INFINITY, m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int t = 0; t < nt; ++t) {
+          int lo, hi;
+          if (geo.is_global(t)) { lo = 0; hi = nvis_i - 1 - t * BN; }
+          else {
+            const int64_t p0 = geo.first(t);
+            lo = int(max(int64_t(-1), c_i - p0));
+            hi = int(min(int64_t(BN), i - p0));
+          }
+          const bool masked = __any_sync(0xffffffffu, lo > 0 || hi < BN - 1);
+          ok = ptx::mbar_wait(&bars[BAR_S + h], uint32_t(t) & 1u, abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          // pass 1: row maximum
+          float mx = -INFINITY;
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            uint32_t v[32];
+            ptx::tmem_ld32(lane_addr + Cfg::colS(h) + c * 32, v);
+            ptx::tc_wait_ld();
+            if (masked) {
+#pragma unroll
+              for (int k = 0; k < 32; ++k) {
+                const int col = c * 32 + k;
+                if (col >= lo && col <= hi) mx = fmaxf(mx, __uint_as_float(v[k]));
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(v[k]));
+            }
+          }
+          m_run = fmaxf(m_run, mx * scale_log2e);
+          // lazy rescale of the accumulator (warp-uniform decision: TMEM access is warp-wide)
+          if (__any_sync(0xffffffffu, m_run > m_used + kRescaleThreshold)) {
+            const float alpha = (m_used == -INFINITY) ? 0.f : ptx::fast_exp2(m_used - m_run);
+            if (t > 0) {
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                ptx::tmem_ld32(lane_addr + Cfg::colO(h) + c * 32, v);
+                ptx::tc_wait_ld();
+#pragma unroll
+                for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * alpha);
+                ptx::tmem_st32(lane_addr + Cfg::colO(h) + c * 32, v);
+              }
+              ptx::tc_wait_st();
+            }
+            l *= alpha;
+            m_used = m_run;
+          }
+          // pass 2: p = exp2(s*scale - m), row sum, bf16 P into swizzled shared memory
+          const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
+          float sum = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            uint32_t v[32];
+            ptx::tmem_ld32(lane_addr + Cfg::colS(h) + c * 32, v);
+            ptx::tc_wait_ld();
+            float p[32];
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              const int col = c * 32 + k;
+              float e = ptx::fast_exp2(fmaf(__uint_as_float(v[k]), scale_log2e, -m_sub));
+              if (masked && (col < lo || col > hi)) e = 0.f;
+              p[k] = e;
+              sum += e;
+            }
+            uint8_t* dst = p_row + (c >> 1) * kHalfBytes;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              uint4 w;
+              w.x = ptx::pack_bf16x2(p[q * 8 + 0], p[q * 8 + 1]);
+              w.y = ptx::pack_bf16x2(p[q * 8 + 2], p[q * 8 + 3]);
+              w.z = ptx::pack_bf16x2(p[q * 8 + 4], p[q * 8 + 5]);
+              w.w = ptx::pack_bf16x2(p[q * 8 + 6], p[q * 8 + 7]);
+              const int chunk = (c & 1) * 4 + q;
+              *reinterpret_cast<uint4*>(dst + ((chunk ^ (row & 7)) << 4)) = w;
+            }
+          }
+          l += sum;
+          ptx::fence_proxy_async_smem();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(&bars[BAR_P + h]);
+        }
+        // epilogue: O / l -> bf16 -> global
+        if (ok) ok = ptx::mbar_wait(&bars[BAR_PV + h], uint32_t(nt - 1) & 1u, abort_flag);
+        if (ok) {
+          ptx::tc_fence_after();
+          const float inv = 1.f / l;
+          __nv_bfloat16* orow = O + (size_t(hq0 + h) * L + size_t(i)) * D;
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t v[32];
+            ptx::tmem_ld32(lane_addr + Cfg::colO(h) + c * 32, v);
+            ptx::tc_wait_ld();
+            if (i <= i_last) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                uint4 w;
+                w.x = ptx::pack_bf16x2(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
+                w.y = ptx::pack_bf16x2(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
+                w.z = ptx::pack_bf16x2(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
+                w.w = ptx::pack_bf16x2(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
+                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = w;
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------- teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (tid == 0) atomicExch(status, 1);
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);  // let copies that are still in flight land
+    __syncthreads();
+  }
+  if (warp == 0) ptx::tmem_dealloc(tmem_base, 512);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// rows x D bf16 matrix (row-major, rows may be a [rows, heads] pair), boxes of 128 rows x 64 columns
+bool encode_map(CUtensorMap* out, const void* base, int D, int64_t rows, int64_t heads, int64_t head_stride_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(rows > 0 ? rows : 1), cuuint64_t(heads)};
+  cuuint64_t strides[2] = {cuuint64_t(D) * 2, cuuint64_t(head_stride_rows) * D * 2};
+  cuuint32_t box[3] = {64, 128, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t rank = heads > 0 ? 3 : 2;
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t prefill_tc_ws_bytes(const tca_params* prm) {
+  const size_t U = size_t(prm->batch) * prm->n_kv_heads;
+  return 256 + (3 + 2 * U) * sizeof(CUtensorMap);
+}
+
+template <int D>
+int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
+                      const tca_cache_desc* c, void* O, void* ws, cudaStream_t stream) {
+  using Cfg = TcCfg<D>;
+  const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
+  const int G = prm->n_q_heads / prm->n_kv_heads;
+  std::vector<CUtensorMap> maps(3 + 2 * U);
+  bool ok = encode_map(&maps[0], Q, D, L, int64_t(prm->batch) * prm->n_q_heads, L) &&
+            encode_map(&maps[1], K, D, L, U, L) && encode_map(&maps[2], V, D, L, U, L);
+  for (int64_t u = 0; u < U && ok; ++u) {
+    const char* kb = static_cast<const char*>(c->k) + size_t(c->seg_start[u]) * D * 2;
+    const char* vb = static_cast<const char*>(c->v) + size_t(c->seg_start[u]) * D * 2;
+    ok = encode_map(&maps[3 + 2 * u], kb, D, c->n_global[u], 0, 0) &&
+         encode_map(&maps[4 + 2 * u], vb, D, c->n_global[u], 0, 0);
+  }
+  if (!ok) return TCA_ERR_CUDA;
+  CUtensorMap* maps_dev = reinterpret_cast<CUtensorMap*>(static_cast<char*>(ws) + 256);
+  // pageable source: staged by the runtime before the call returns
+  TCA_CHECK_CUDA(cudaMemcpyAsync(maps_dev, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice,
+                                 stream));
+  auto kern = prefill_tc_kernel<D>;
+  TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::bytes));
+  const int n_qtiles = int((L + BM - 1) / BM);
+  const int pairs = (G + 1) / 2;
+  const int64_t n_ctas = int64_t(n_qtiles) * U * pairs;
+  if (n_ctas >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;
+  const int64_t mb = num_blocks(prm, L) * prm->block;
+  kern<<<unsigned(n_ctas), kThreads, Cfg::bytes, stream>>>(
+      maps_dev, c->pos, c->state, L, prm->n_q_heads, prm->n_kv_heads, prm->window, mb,
+      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs);
+  return check_launch();
+}
+
+template int launch_prefill_tc<64>(const tca_params*, const void*, const void*, const void*, int64_t,
+                                   const tca_cache_desc*, void*, void*, cudaStream_t);
+template int launch_prefill_tc<128>(const tca_params*, const void*, const void*, const void*, int64_t,
+                                    const tca_cache_desc*, void*, void*, cudaStream_t);
+
+}  // namespace tca
