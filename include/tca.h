@@ -161,7 +161,8 @@ int tca_select(const tca_params* prm, const double* logscore, int64_t L,
                double* h_out, int32_t* t_out, void* ws, size_t ws_bytes, void* stream);
 
 /* Upload the host mirror of `cache` (seg_start, global_cap, n_global, tail_head, n_tail,
- * seq_len, t_keep) into cache->state.  Call once after filling the descriptor. */
+ * seq_len, t_keep) into cache->state and zero-fill cache->k and cache->v (rows that are
+ * not in use must hold finite values).  Call once after filling the descriptor. */
 int tca_cache_init(const tca_params* prm, tca_cache_desc* cache, void* stream);
 
 /*
@@ -193,7 +194,9 @@ int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const 
  * One decode step, Eq. 2 with a single query per head over the whole retained cache
  * (global region + tail ring) of its KV head.
  *   q  DEVICE [batch, n_q_heads, head_dim]     O  DEVICE out, same shape
- *   ws DEVICE workspace, tca_workspace_bytes(prm, cache->rows_total, TCA_OP_DECODE)
+ *   ws DEVICE workspace, tca_workspace_bytes(prm, cache->rows_total, TCA_OP_DECODE).  Its
+ *      first word is a sticky error flag (tca_ws_status): zero it once after allocating;
+ *      a kernel sets it if one of its bounded waits gave up, and never clears it.
  */
 int tca_attn_decode(const tca_params* prm, const void* q, const tca_cache_desc* cache,
                     void* O, void* ws, size_t ws_bytes, void* stream);

@@ -129,11 +129,13 @@ def _ws_args(ws: Optional[torch.Tensor]):
 
 
 def alloc_workspace(prm: tca_params, L: int, op: int, device="cuda") -> torch.Tensor:
-    """A device buffer of tca_workspace_bytes(prm, L, op) bytes (torch owns the memory)."""
+    """A zero-filled device buffer of tca_workspace_bytes(prm, L, op) bytes (torch owns the
+    memory).  Zero-filled because the first word of the prefill and decode workspaces is a
+    sticky error flag that tca_ws_status reads."""
     n = tca_workspace_bytes(prm, L, op)
     if n == 0:
         raise TcaError(TCA_ERR_INVALID_ARG, "tca_workspace_bytes")
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    return torch.zeros(n, dtype=torch.uint8, device=device)
 
 
 # ----------------------------------------------------------------------------- the C entry points

@@ -53,10 +53,11 @@ SelectWs select_ws_layout(const tca_params* prm, int64_t L, void* ws) {
 DecodeWs decode_ws_layout(const tca_params* prm, int64_t rows_total, int64_t n_units, void* ws) {
   DecodeWs w;
   const int G = prm->n_q_heads / prm->n_kv_heads;
-  // every unit wastes at most one partially filled chunk per region (global, ring)
+  // slices are at least kDecodeChunkRows long, plus one short slice per unit
   w.n_chunks_max = rows_total / kDecodeChunkRows + 2 * n_units + 1;
-  w.partial = reinterpret_cast<float*>(ws);
-  w.bytes = align_up(size_t(w.n_chunks_max) * G * (prm->head_dim + 2) * sizeof(float), 256);
+  w.status = reinterpret_cast<int*>(ws);
+  w.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + 256);
+  w.bytes = 256 + align_up(size_t(w.n_chunks_max) * G * (prm->head_dim + 2) * sizeof(float), 256);
   return w;
 }
 
@@ -171,6 +172,11 @@ int tca_cache_init(const tca_params* prm, tca_cache_desc* c, void* stream) {
     s[TCA_ST_SEQ_LEN] = c->seq_len[u];
     s[TCA_ST_T_KEEP] = c->t_keep[u];
   }
+  // Unused rows must hold finite values: the tensor-pipe kernels multiply masked-out rows by
+  // an exact zero weight, which only cancels finite numbers.
+  const size_t cache_bytes = size_t(c->rows_total) * prm->head_dim * elt_size(prm->dtype);
+  TCA_CHECK_CUDA(cudaMemsetAsync(c->k, 0, cache_bytes, static_cast<cudaStream_t>(stream)));
+  TCA_CHECK_CUDA(cudaMemsetAsync(c->v, 0, cache_bytes, static_cast<cudaStream_t>(stream)));
   // pageable source: the runtime stages the bytes before returning, so the vector may die
   TCA_CHECK_CUDA(cudaMemcpyAsync(c->state, st_host.data(), st_host.size() * sizeof(int64_t),
                                  cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));

@@ -62,9 +62,11 @@ struct SelectWs {
 };
 SelectWs select_ws_layout(const tca_params* prm, int64_t L, void* ws);
 
-// decode: partial (m, l, acc[d]) per (chunk, query head of the group).
-constexpr int kDecodeChunkRows = 256;  // cache rows per CTA of the split-KV kernel
+// decode: a 256-byte header (word 0: sticky error flag, set when a bounded wait gave up)
+// followed by one partial (acc[d], max, sum) per (slice, query head of the group).
+constexpr int kDecodeChunkRows = 256;  // smallest slice of cache rows one CTA takes
 struct DecodeWs {
+  int* status;
   float* partial;     // [n_chunks_max][G][d + 2]
   int64_t n_chunks_max;
   size_t bytes;

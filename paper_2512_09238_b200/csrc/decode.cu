@@ -2,192 +2,259 @@
 // (Eq. 2 at decode time; HBM-bound: every retained K and V row is read exactly once per
 // step and shared by the G query heads of the group).
 //
-//   decode_split_kernel   CTA = (chunk of kDecodeChunkRows cache rows, unit).  Phase A
-//                         streams the chunk's K rows (16 lanes x 16 B per row), forms the
-//                         G logits per row with a transposing shuffle butterfly and parks
-//                         them in shared memory; the chunk maximum and exp2 follow; phase B
-//                         streams the V rows and accumulates p*V per lane slice.  Writes an
-//                         un-normalised partial (acc, max, sum) per (chunk, query head).
-//   decode_combine_kernel merges a unit's partials in chunk order (fixed order => bit-
+//   decode_split_kernel   CTA = (slice of a unit's cache rows, unit); the rows of all units are cut
+//                         into about two slices per SM.  A producer warp streams the slice's K and
+//                         V rows through a shared-memory ring of 64-row tiles with 1-D bulk
+//                         asynchronous copies (up to 96 KB in flight per CTA, independent of the
+//                         consumers' registers).  Eight consumer warps work in rounds of 256 rows:
+//                         K phase (G logits per row by a transposing shuffle butterfly, parked in
+//                         shared memory), running maximum + exp2, V phase (p*V per lane slice).
+//                         Writes one un-normalised partial (acc, max, sum) per (slice, query head).
+//   decode_combine_kernel merges a unit's partials in slice order (fixed order => bit-
 //                         reproducible) and normalises.
 #include <mutex>
 
+#include "bulk_ring.cuh"
 #include "common.cuh"
+#include "decode_common.cuh"
 #include "rowslice.cuh"
 
 namespace tca {
+
+template <int D>
+int launch_decode_mma(const tca_params*, const void*, const tca_cache_desc*, const DecodeWs&, int64_t, int,
+                      cudaStream_t);
+
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kGroups = kThreads / 16;
-constexpr int CH = kDecodeChunkRows;
+constexpr int kConsumers = 256;              // 8 consumer warps
+constexpr int kThreads = kConsumers + 32;    // + 1 producer warp
+constexpr int kGroups = kConsumers / 16;     // 16-lane groups, one cache row each
+constexpr int kTileRows = 64;                // rows per ring tile (4 per lane group)
+constexpr int kSuperRows = 256;              // rows per softmax round (4 tiles)
+constexpr int kRingBytes = 96 * 1024;
 
 template <int G>
 struct DecCfg {
-  static constexpr int R = (G == 1) ? 16 : (G == 2) ? 8 : 4;
+  static constexpr int R = 4;                // rows per lane group per tile
   static constexpr int NV = R * G;
   static constexpr int NB = (NV + 15) / 16;
   static constexpr int NVP = NB * 16;
 };
 
-struct UnitView {
-  int64_t seg, gcap, n_global, tail_head, n_tail, tail_cap;
-  __device__ __forceinline__ int64_t len() const { return n_global + n_tail; }
-  // logical row (global rows first, then the tail oldest-first) -> physical cache row
-  __device__ __forceinline__ int64_t phys(int64_t r) const {
-    if (r < n_global) return seg + r;
-    int64_t slot = tail_head + (r - n_global);
-    if (slot >= tail_cap) slot -= tail_cap;
-    return seg + gcap + slot;
-  }
+template <typename T, int D>
+struct DecRing {
+  static constexpr int kTileBytes = kTileRows * D * int(sizeof(T));
+  static constexpr int kStages = kRingBytes / kTileBytes > 8 ? 8 : kRingBytes / kTileBytes;
+  static constexpr int kSmemBytes = kStages * kTileBytes + 1024;
 };
 
-__device__ __forceinline__ UnitView load_unit(const int64_t* state, int u, int64_t tail_cap) {
-  const int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
-  UnitView v;
-  v.seg = st[TCA_ST_SEG_START];
-  v.gcap = st[TCA_ST_GLOBAL_CAP];
-  v.n_global = st[TCA_ST_N_GLOBAL];
-  v.tail_head = st[TCA_ST_TAIL_HEAD];
-  v.n_tail = st[TCA_ST_N_TAIL];
-  v.tail_cap = tail_cap;
-  return v;
-}
-
-__device__ __forceinline__ int64_t partial_base(const UnitView& v, int u) {
-  return v.seg / CH + 2 * int64_t(u);
-}
-
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* __restrict__ Vc,
-                    const int64_t* __restrict__ state, int64_t tail_cap, float scale_log2e,
-                    float* __restrict__ partial) {
+                    const int64_t* __restrict__ state, int64_t tail_cap, float scale_log2e, int target,
+                    float* __restrict__ partial, int* __restrict__ status) {
   using Cfg = DecCfg<G>;
+  using Ring = DecRing<T, D>;
   constexpr int EPL = D / 16;
   constexpr int R = Cfg::R, NB = Cfg::NB;
+  constexpr int kStages = Ring::kStages;
   const int u = blockIdx.y;
-  const int chunk = blockIdx.x;
+  const int part_idx = blockIdx.x;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int64_t len = uv.len();
-  const int64_t row0 = int64_t(chunk) * CH;
-  if (row0 >= len) return;
-  const int n_rows = int(min(int64_t(CH), len - row0));
+  if (part_idx >= n_parts(len, target)) return;
+  const int64_t row0 = int64_t(part_idx) * target;
+  const int n_rows = int(min(int64_t(target), len - row0));
+  const int n_super = (n_rows + kSuperRows - 1) / kSuperRows;
   const int tid = threadIdx.x, lane16 = tid & 15, grp = tid >> 4, warp = tid >> 5;
+  const int base_slot = partial_base<kThreads>(state, u, target);
 
-  __shared__ float xs[CH][G];
-  __shared__ float red[kThreads / 32][G][D];
-  __shared__ float stat_m[G], stat_l[G];
-  __shared__ float wred[kThreads / 32][G];
+  extern __shared__ uint8_t dec_smem_raw[];
+  uint8_t* ring_buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dec_smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ BulkRing<kStages> ring;
+  __shared__ int abort_word;
+  __shared__ float xs[kSuperRows][G];
+  __shared__ float stat_m[G], stat_c[G], stat_l[G];
+  __shared__ float wred[kConsumers / 32][G];
+  volatile int* abort_flag = &abort_word;
+  if (tid == 0) {
+    ring.init(kConsumers / 32);   // one release per consumer warp
+    abort_word = 0;
+  }
+  if (tid < G) { stat_m[tid] = -INFINITY; stat_l[tid] = 0.f; }
+  __syncthreads();
 
+  if (warp == kConsumers / 32) {
+    // ------------------------------------------------------------- producer: K tiles then V tiles of every round
+    if ((tid & 31) == 0) {
+      int n = 0;
+      for (int s = 0; s < n_super; ++s) {
+        const int srow = s * kSuperRows;
+        const int rows_here = min(kSuperRows, n_rows - srow);
+        const int tiles = (rows_here + kTileRows - 1) / kTileRows;
+        for (int kv = 0; kv < 2; ++kv) {
+          const T* src = kv ? Vc : Kc;
+          for (int k = 0; k < tiles; ++k, ++n) {
+            const int trow = srow + k * kTileRows;
+            const int cnt = min(kTileRows, n_rows - trow);
+            if (!ring.acquire(n, uint32_t(cnt) * D * sizeof(T), abort_flag)) return;
+            uint8_t* dst = ring_buf + (n % kStages) * Ring::kTileBytes;
+            int done = 0;
+            while (done < cnt) {   // at most three physically contiguous runs
+              const int64_t r = row0 + trow + done;
+              const int run = int(uv.run(r, cnt - done));
+              bulk_copy_g2s(dst + size_t(done) * D * sizeof(T), src + size_t(uv.phys(r)) * D,
+                            uint32_t(run) * D * sizeof(T), &ring.full[n % kStages]);
+              done += run;
+            }
+          }
+        }
+      }
+    }
+    return;
+  }
+
+  // --------------------------------------------------------------- consumers
   float qf[G][EPL];
 #pragma unroll
   for (int g = 0; g < G; ++g)
 #pragma unroll
     for (int e = 0; e < EPL; ++e)
       qf[g][e] = elt_to_float(q[(size_t(u) * G + g) * D + lane16 * EPL + e]) * scale_log2e;
-
-  // ---- phase A: logits (in log2 units) of every row of the chunk
-  for (int base = 0; base < CH; base += kGroups * R) {
-    RowF<T, EPL> raw[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const int lr = base + r * kGroups + grp;
-      if (lr < n_rows) raw[r].load(Kc + size_t(uv.phys(row0 + lr)) * D + lane16 * EPL);
-      else raw[r].zero();
-    }
-    float acc[Cfg::NVP];
-#pragma unroll
-    for (int i = 0; i < Cfg::NVP; ++i) acc[i] = 0.f;
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        const float kf = raw[r].get(e);
-#pragma unroll
-        for (int g = 0; g < G; ++g) acc[r * G + g] = fmaf(qf[g][e], kf, acc[r * G + g]);
-      }
-#pragma unroll
-    for (int bf = 0; bf < NB; ++bf) {
-      float part[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) part[i] = acc[bf * 16 + i];
-      const float x = butterfly16f(part, lane16);
-      const int v = bf * 16 + lane16;
-      const int r = v / G, g = v - r * G;
-      const int lr = base + r * kGroups + grp;
-      if (v < Cfg::NV && lr < CH) xs[lr][g] = (lr < n_rows) ? x : -INFINITY;
-    }
-  }
-  __syncthreads();
-
-  // ---- chunk maximum, exponentials and their sum, per query head (thread = row)
-  {
-    float xv[G];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      xv[g] = xs[tid][g];
-      float mx = xv[g];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-      if ((tid & 31) == 0) wred[warp][g] = mx;
-    }
-    __syncthreads();
-    if (tid < G) {
-      float mx = wred[0][tid];
-      for (int w = 1; w < kThreads / 32; ++w) mx = fmaxf(mx, wred[w][tid]);
-      stat_m[tid] = mx;
-    }
-    __syncthreads();
-    float pv[G];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      pv[g] = exp2f(xv[g] - stat_m[g]);
-      xs[tid][g] = pv[g];
-      float sum = pv[g];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-      if ((tid & 31) == 0) wred[warp][g] = sum;
-    }
-    __syncthreads();
-    if (tid < G) {
-      float sum = 0.f;
-      for (int w = 0; w < kThreads / 32; ++w) sum += wred[w][tid];
-      stat_l[tid] = sum;
-    }
-  }
-  __syncthreads();
-
-  // ---- phase B: acc[g][e] += p[row][g] * V[row][e]
   float o[G][EPL];
 #pragma unroll
   for (int g = 0; g < G; ++g)
 #pragma unroll
     for (int e = 0; e < EPL; ++e) o[g][e] = 0.f;
-  constexpr int RB = 4;
-  for (int base = 0; base < n_rows; base += kGroups * RB) {
-    RowF<T, EPL> raw[RB];
+
+  int n = 0;
+  bool ok = true;
+  // A wait that gives up clears `ok`; the thread then skips the work but still walks the same
+  // barriers as everybody else, so nobody is left waiting at a barrier.
+  for (int s = 0; s < n_super; ++s) {
+    const int srow = s * kSuperRows;
+    const int rows_here = min(kSuperRows, n_rows - srow);
+    const int tiles = (rows_here + kTileRows - 1) / kTileRows;
+    // ---- phase A: logits (log2 units) of the round's rows
+    for (int k = 0; k < tiles; ++k, ++n) {
+      if (ok) ok = ring.wait_full(n, abort_flag);
+      if (!ok) continue;
+      const T* tile = reinterpret_cast<const T*>(ring_buf + (n % kStages) * Ring::kTileBytes);
+      RowF<T, EPL> raw[R];
 #pragma unroll
-    for (int r = 0; r < RB; ++r) {
-      const int lr = base + r * kGroups + grp;
-      if (lr < n_rows) raw[r].load(Vc + size_t(uv.phys(row0 + lr)) * D + lane16 * EPL);
-      else raw[r].zero();
-    }
+      for (int r = 0; r < R; ++r) {
+        const int tr = r * kGroups + grp;                   // row inside the tile
+        if (k * kTileRows + tr < rows_here) raw[r].load_cached(tile + size_t(tr) * D + lane16 * EPL);
+        else raw[r].zero();
+      }
+      __syncwarp();
+      if ((tid & 31) == 0) ring.release(n);
+      float acc[Cfg::NVP];
 #pragma unroll
-    for (int r = 0; r < RB; ++r) {
-      const int lr = min(base + r * kGroups + grp, CH - 1);
-      float p[G];
+      for (int i = 0; i < Cfg::NVP; ++i) acc[i] = 0.f;
 #pragma unroll
-      for (int g = 0; g < G; ++g) p[g] = xs[lr][g];
+      for (int r = 0; r < R; ++r)
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        const float vf = raw[r].get(e);
+        for (int e = 0; e < EPL; ++e) {
+          const float kf = raw[r].get(e);
 #pragma unroll
-        for (int g = 0; g < G; ++g) o[g][e] = fmaf(p[g], vf, o[g][e]);
+          for (int g = 0; g < G; ++g) acc[r * G + g] = fmaf(qf[g][e], kf, acc[r * G + g]);
+        }
+#pragma unroll
+      for (int bf = 0; bf < NB; ++bf) {
+        float part[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) part[i] = acc[bf * 16 + i];
+        const float x = butterfly16f(part, lane16);
+        const int v = bf * 16 + lane16;
+        const int r = v / G, g = v - r * G;
+        const int lr = k * kTileRows + r * kGroups + grp;
+        if (v < Cfg::NV) xs[lr][g] = (lr < rows_here) ? x : -INFINITY;
       }
     }
+    consumer_sync(kConsumers);
+    // ---- running maximum, exponentials and their sum, per query head (thread = row)
+    {
+      const bool live = tid < tiles * kTileRows;
+      float xv[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        xv[g] = live ? xs[tid][g] : -INFINITY;
+        float mx = xv[g];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        if ((tid & 31) == 0) wred[warp][g] = mx;
+      }
+      consumer_sync(kConsumers);
+      if (tid < G) {
+        float mx = stat_m[tid];
+        const float old = mx;
+        for (int w = 0; w < kConsumers / 32; ++w) mx = fmaxf(mx, wred[w][tid]);
+        stat_c[tid] = (old == -INFINITY) ? 0.f : exp2f(old - mx);
+        stat_m[tid] = mx;
+      }
+      consumer_sync(kConsumers);
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float pv = exp2f(xv[g] - stat_m[g]);
+        if (live) xs[tid][g] = pv;
+        float sum = pv;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if ((tid & 31) == 0) wred[warp][g] = sum;
+      }
+      consumer_sync(kConsumers);
+      if (tid < G) {
+        float sum = 0.f;
+        for (int w = 0; w < kConsumers / 32; ++w) sum += wred[w][tid];
+        stat_l[tid] = stat_l[tid] * stat_c[tid] + sum;
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float c = stat_c[g];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) o[g][e] *= c;
+      }
+    }
+    // ---- phase B: acc[g][e] += p[row][g] * V[row][e]
+    for (int k = 0; k < tiles; ++k, ++n) {
+      if (ok) ok = ring.wait_full(n, abort_flag);
+      if (!ok) continue;
+      const T* tile = reinterpret_cast<const T*>(ring_buf + (n % kStages) * Ring::kTileBytes);
+      RowF<T, EPL> raw[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int tr = r * kGroups + grp;
+        if (k * kTileRows + tr < rows_here) raw[r].load_cached(tile + size_t(tr) * D + lane16 * EPL);
+        else raw[r].zero();
+      }
+      __syncwarp();
+      if ((tid & 31) == 0) ring.release(n);
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int lr = k * kTileRows + r * kGroups + grp;
+        float p[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) p[g] = (lr < rows_here) ? xs[lr][g] : 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          const float vf = raw[r].get(e);
+#pragma unroll
+          for (int g = 0; g < G; ++g) o[g][e] = fmaf(p[g], vf, o[g][e]);
+        }
+      }
+    }
+    consumer_sync(kConsumers);   // xs is rewritten by the next round
   }
+  if (*abort_flag) {   // uniform after the barrier above: some wait gave up, the result is not valid
+    if (tid == 0) atomicExch(status, 1);
+    return;
+  }
+
   // the two 16-lane groups of a warp, then the warps, in a fixed order
+  float(*red)[G][D] = reinterpret_cast<float(*)[G][D]>(ring_buf);   // the ring is drained: reuse it
+  static_assert(sizeof(float) * (kConsumers / 32) * G * D <= size_t(Ring::kStages) * Ring::kTileBytes, "ring too small");
 #pragma unroll
   for (int g = 0; g < G; ++g)
 #pragma unroll
@@ -198,13 +265,13 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
 #pragma unroll
       for (int e = 0; e < EPL; ++e) red[warp][g][lane16 * EPL + e] = o[g][e];
   }
-  __syncthreads();
-  float* out = partial + size_t(partial_base(uv, u) + chunk) * G * (D + 2);
-  for (int i = tid; i < G * D; i += kThreads) {
+  consumer_sync(kConsumers);
+  float* out = partial + size_t(base_slot + part_idx) * G * (D + 2);
+  for (int i = tid; i < G * D; i += kConsumers) {
     const int g = i / D, d = i - g * D;
     float sum = 0.f;
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) sum += red[w][g][d];
+    for (int w = 0; w < kConsumers / 32; ++w) sum += red[w][g][d];
     out[size_t(g) * (D + 2) + d] = sum;
   }
   if (tid < G) {
@@ -216,73 +283,122 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads)
 decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restrict__ state, int64_t tail_cap,
-                      T* __restrict__ O) {
-  constexpr int NCL = kThreads / D;  // chunk lanes
+                      int target, T* __restrict__ O) {
+  constexpr int NW = kConsumers / 32;   // warp w merges partials w, w + NW, ...; a lane owns 4 outputs
   const int g = blockIdx.x, u = blockIdx.y;
   const UnitView uv = load_unit(state, u, tail_cap);
-  const int n_chunks = int((uv.len() + CH - 1) / CH);
-  const float* base = partial + size_t(partial_base(uv, u)) * G * (D + 2) + size_t(g) * (D + 2);
+  const int n_chunks = n_parts(uv.len(), target);
+  const int base_slot = partial_base<kThreads>(state, u, target);
+  const int tid = threadIdx.x;
+  if (tid >= kConsumers) return;
+  const float* base = partial + size_t(base_slot) * G * (D + 2) + size_t(g) * (D + 2);
   const size_t stride = size_t(G) * (D + 2);
-  const int tid = threadIdx.x, d = tid % D, cl = tid / D;
-  __shared__ float s_max[kThreads / 32];
-  __shared__ float s_acc[NCL][D], s_l[NCL];
+  const int warp = tid >> 5, lane = tid & 31;
+  __shared__ float s_max[NW];
+  __shared__ float s_acc[NW][D], s_l[NW];
 
   float mx = -INFINITY;
-  for (int c = tid; c < n_chunks; c += kThreads) mx = fmaxf(mx, base[c * stride + D]);
+  for (int c = tid; c < n_chunks; c += kConsumers) mx = fmaxf(mx, base[c * stride + D]);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-  if ((tid & 31) == 0) s_max[tid >> 5] = mx;
-  __syncthreads();
+  if (lane == 0) s_max[warp] = mx;
+  consumer_sync(kConsumers);
   mx = s_max[0];
 #pragma unroll
-  for (int w = 1; w < kThreads / 32; ++w) mx = fmaxf(mx, s_max[w]);
+  for (int w = 1; w < NW; ++w) mx = fmaxf(mx, s_max[w]);
 
-  float acc = 0.f, l = 0.f;
-  for (int c = cl; c < n_chunks; c += NCL) {
+  // independent loads of up to four partials are in flight per lane
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float l = 0.f;
+  const bool owns = lane * 4 < D;
+#pragma unroll 4
+  for (int c = warp; c < n_chunks; c += NW) {
     const float* p = base + c * stride;
     const float w = exp2f(p[D] - mx);
-    acc = fmaf(p[d], w, acc);
     l = fmaf(p[D + 1], w, l);
+    if (owns) {
+      const float2 a = *reinterpret_cast<const float2*>(p + lane * 4);
+      const float2 b = *reinterpret_cast<const float2*>(p + lane * 4 + 2);
+      acc[0] = fmaf(a.x, w, acc[0]);
+      acc[1] = fmaf(a.y, w, acc[1]);
+      acc[2] = fmaf(b.x, w, acc[2]);
+      acc[3] = fmaf(b.y, w, acc[3]);
+    }
   }
-  s_acc[cl][d] = acc;
-  if (d == 0) s_l[cl] = l;
-  __syncthreads();
-  if (cl == 0) {
+  if (owns) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s_acc[warp][lane * 4 + i] = acc[i];
+  }
+  if (lane == 0) s_l[warp] = l;
+  consumer_sync(kConsumers);
+  if (tid < D) {
     float a = 0.f, ls = 0.f;
 #pragma unroll
-    for (int i = 0; i < NCL; ++i) { a += s_acc[i][d]; ls += s_l[i]; }
-    store_elt(O + (size_t(u) * G + g) * D + d, n_chunks > 0 ? a / ls : 0.f);
+    for (int w = 0; w < NW; ++w) { a += s_acc[w][tid]; ls += s_l[w]; }
+    store_elt(O + (size_t(u) * G + g) * D + tid, n_chunks > 0 ? a / ls : 0.f);
   }
+}
+
+// Rows per CTA: enough CTAs for two per SM, at least one softmax round each.
+inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_sm, int64_t* max_len_out) {
+  int64_t total = 0, max_len = 0;
+  for (int64_t u = 0; u < U; ++u) {
+    const int64_t len = c->n_global[u] + c->n_tail[u];
+    total += len;
+    max_len = len > max_len ? len : max_len;
+  }
+  *max_len_out = max_len;
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      sms = n;
+    else
+      sms = 148;
+  }
+  int64_t target = (total + ctas_per_sm * sms - 1) / (ctas_per_sm * sms);
+  target = (target + kTileRows - 1) / kTileRows * kTileRows;
+  if (target < kSuperRows) target = kSuperRows;
+  return int(target);
 }
 
 template <typename T, int D, int G>
 int launch_decode(const tca_params* prm, const void* q, const tca_cache_desc* c, void* O, const DecodeWs& ws,
-                  int64_t max_len, cudaStream_t stream) {
+                  int64_t max_len, int target, cudaStream_t stream) {
+  using Ring = DecRing<T, D>;
   const int U = prm->batch * prm->n_kv_heads;
   const float scale_log2e = prm->sm_scale * 1.4426950408889634f;
-  dim3 grid(unsigned((max_len + CH - 1) / CH), unsigned(U));
-  decode_split_kernel<T, D, G><<<grid, kThreads, 0, stream>>>(
-      static_cast<const T*>(q), static_cast<const T*>(c->k), static_cast<const T*>(c->v), c->state,
-      c->tail_cap, scale_log2e, ws.partial);
-  int st = check_launch();
+  auto kern = decode_split_kernel<T, D, G>;
+  TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Ring::kSmemBytes));
+  int st;
+  if constexpr (sizeof(T) == 2) {
+    st = launch_decode_mma<D>(prm, q, c, ws, max_len, target, stream);   // tensor-pipe kernel for bf16
+  } else {
+    dim3 grid(unsigned((max_len + target - 1) / target), unsigned(U));
+    kern<<<grid, kThreads, Ring::kSmemBytes, stream>>>(
+        static_cast<const T*>(q), static_cast<const T*>(c->k), static_cast<const T*>(c->v), c->state,
+        c->tail_cap, scale_log2e, target, ws.partial, ws.status);
+    st = check_launch();
+  }
   if (st != TCA_OK) return st;
   decode_combine_kernel<T, D, G><<<dim3(G, unsigned(U)), kThreads, 0, stream>>>(ws.partial, c->state, c->tail_cap,
-                                                                               static_cast<T*>(O));
+                                                                               target, static_cast<T*>(O));
   return check_launch();
 }
 
 template <typename T, int D>
 int dispatch_group(int G, const tca_params* prm, const void* q, const tca_cache_desc* c, void* O,
-                   const DecodeWs& ws, int64_t max_len, cudaStream_t s) {
+                   const DecodeWs& ws, int64_t max_len, int target, cudaStream_t s) {
   switch (G) {
-    case 1: return launch_decode<T, D, 1>(prm, q, c, O, ws, max_len, s);
-    case 2: return launch_decode<T, D, 2>(prm, q, c, O, ws, max_len, s);
-    case 3: return launch_decode<T, D, 3>(prm, q, c, O, ws, max_len, s);
-    case 4: return launch_decode<T, D, 4>(prm, q, c, O, ws, max_len, s);
-    case 5: return launch_decode<T, D, 5>(prm, q, c, O, ws, max_len, s);
-    case 6: return launch_decode<T, D, 6>(prm, q, c, O, ws, max_len, s);
-    case 7: return launch_decode<T, D, 7>(prm, q, c, O, ws, max_len, s);
-    case 8: return launch_decode<T, D, 8>(prm, q, c, O, ws, max_len, s);
+    case 1: return launch_decode<T, D, 1>(prm, q, c, O, ws, max_len, target, s);
+    case 2: return launch_decode<T, D, 2>(prm, q, c, O, ws, max_len, target, s);
+    case 3: return launch_decode<T, D, 3>(prm, q, c, O, ws, max_len, target, s);
+    case 4: return launch_decode<T, D, 4>(prm, q, c, O, ws, max_len, target, s);
+    case 5: return launch_decode<T, D, 5>(prm, q, c, O, ws, max_len, target, s);
+    case 6: return launch_decode<T, D, 6>(prm, q, c, O, ws, max_len, target, s);
+    case 7: return launch_decode<T, D, 7>(prm, q, c, O, ws, max_len, target, s);
+    case 8: return launch_decode<T, D, 8>(prm, q, c, O, ws, max_len, target, s);
     default: return TCA_ERR_UNSUPPORTED;
   }
 }
@@ -304,19 +420,16 @@ extern "C" int tca_attn_decode(const tca_params* prm, const void* q, const tca_c
   DecodeWs lay = decode_ws_layout(prm, c->rows_total, U, ws);
   if (ws_bytes < lay.bytes) return TCA_ERR_WORKSPACE;
   int64_t max_len = 0;
-  for (int64_t u = 0; u < U; ++u) {
-    const int64_t len = c->n_global[u] + c->n_tail[u];
-    max_len = len > max_len ? len : max_len;
-  }
+  const int target = decode_target_rows(c, U, prm->dtype == TCA_BF16 ? 1 : 2, &max_len);
   TCA_CHECK_ARG(max_len >= 1);
   const int G = prm->n_q_heads / prm->n_kv_heads;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (prm->dtype == TCA_BF16) {
-    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, s);
-    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, s);
+    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, target, s);
+    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, target, s);
   }
-  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, s);
-  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, s);
+  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, target, s);
+  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, target, s);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -370,17 +483,14 @@ extern "C" int tca_attn_decode_static(const tca_params* prm, const void* q, cons
   if (st != TCA_OK) return st;
   lay = decode_ws_layout(prm, c->rows_total, U, scratch);
   int64_t max_len = 0;
-  for (int64_t u = 0; u < U; ++u) {
-    const int64_t len = c->n_global[u] + c->n_tail[u];
-    max_len = len > max_len ? len : max_len;
-  }
+  const int target = decode_target_rows(c, U, prm->dtype == TCA_BF16 ? 1 : 2, &max_len);
   TCA_CHECK_ARG(max_len >= 1);
   const int G = prm->n_q_heads / prm->n_kv_heads;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (prm->dtype == TCA_BF16) {
-    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, s);
-    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, s);
+    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, target, s);
+    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, target, s);
   }
-  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, s);
-  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, s);
+  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, target, s);
+  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, target, s);
 }

@@ -1,0 +1,63 @@
+// Pieces shared by the decode kernels: the view of a unit's cache segment, the slicing of
+// its rows over CTAs and the packing of the per-slice partial results.
+#pragma once
+#include "common.cuh"
+
+namespace tca {
+
+struct UnitView {
+  int64_t seg, gcap, n_global, tail_head, n_tail, tail_cap;
+  __device__ __forceinline__ int64_t len() const { return n_global + n_tail; }
+  // logical row (global rows first, then the tail oldest-first) -> physical cache row
+  __device__ __forceinline__ int64_t phys(int64_t r) const {
+    if (r < n_global) return seg + r;
+    int64_t slot = tail_head + (r - n_global);
+    if (slot >= tail_cap) slot -= tail_cap;
+    return seg + gcap + slot;
+  }
+  // rows [r, r+n) are physically contiguous for the returned count (<= n)
+  __device__ __forceinline__ int64_t run(int64_t r, int64_t n) const {
+    if (r < n_global) return min(n, n_global - r);
+    int64_t slot = tail_head + (r - n_global);
+    if (slot >= tail_cap) slot -= tail_cap;
+    return min(n, tail_cap - slot);
+  }
+};
+
+__device__ __forceinline__ UnitView load_unit(const int64_t* state, int u, int64_t tail_cap) {
+  const int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
+  UnitView v;
+  v.seg = st[TCA_ST_SEG_START];
+  v.gcap = st[TCA_ST_GLOBAL_CAP];
+  v.n_global = st[TCA_ST_N_GLOBAL];
+  v.tail_head = st[TCA_ST_TAIL_HEAD];
+  v.n_tail = st[TCA_ST_N_TAIL];
+  v.tail_cap = tail_cap;
+  return v;
+}
+
+// CTAs of unit u: ceil(len / target).  Partials are packed unit after unit.
+__device__ __forceinline__ int n_parts(int64_t len, int target) { return int((len + target - 1) / target); }
+
+template <int kBlockThreads>
+__device__ __forceinline__ int partial_base(const int64_t* state, int u, int target) {
+  // sum of n_parts over the units before u (all threads of the CTA call this together)
+  __shared__ int s_base[kBlockThreads / 32];
+  int part = 0;
+  for (int v = threadIdx.x; v < u; v += kBlockThreads) {
+    const int64_t* st = state + size_t(v) * TCA_STATE_WORDS;
+    part += n_parts(st[TCA_ST_N_GLOBAL] + st[TCA_ST_N_TAIL], target);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+  if ((threadIdx.x & 31) == 0) s_base[threadIdx.x >> 5] = part;
+  __syncthreads();
+  int total = 0;
+#pragma unroll
+  for (int w = 0; w < kBlockThreads / 32; ++w) total += s_base[w];
+  __syncthreads();
+  return total;
+}
+
+
+}  // namespace tca
