@@ -50,7 +50,7 @@ struct DecRing {
 };
 
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __maxnreg__(112)
 decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* __restrict__ Vc,
                     const int64_t* __restrict__ state, int64_t tail_cap, float scale_log2e, int target,
                     float* __restrict__ partial, int* __restrict__ status) {

@@ -33,7 +33,7 @@ struct RowSlice<__nv_bfloat16, 8> {
   __device__ __forceinline__ void zero() { raw = make_uint4(0, 0, 0, 0); }
   __device__ __forceinline__ double get(int e) const {
     uint32_t w = (e < 2) ? raw.x : (e < 4) ? raw.y : (e < 6) ? raw.z : raw.w;
-    return bf16_bits_to_double((e & 1) ? (w >> 16) : (w & 0xFFFFu));
+    return (e & 1) ? bf16_hi_to_double(w) : bf16_lo_to_double(w);
   }
 };
 template <>
@@ -43,7 +43,7 @@ struct RowSlice<__nv_bfloat16, 4> {
   __device__ __forceinline__ void zero() { raw = make_uint2(0, 0); }
   __device__ __forceinline__ double get(int e) const {
     uint32_t w = (e < 2) ? raw.x : raw.y;
-    return bf16_bits_to_double((e & 1) ? (w >> 16) : (w & 0xFFFFu));
+    return (e & 1) ? bf16_hi_to_double(w) : bf16_lo_to_double(w);
   }
 };
 template <>
@@ -274,7 +274,7 @@ int launch_score(const tca_params* prm, const void* q_last, const void* K, int64
       ws.partials, int(ws.n_chunks));
   int st = check_launch();
   if (st != TCA_OK) return st;
-  const int rows_per_cta = 2048;
+  const int rows_per_cta = 1024;
   dim3 grid2(unsigned((L + rows_per_cta - 1) / rows_per_cta), unsigned(U));
   score_finalize_kernel<G><<<grid2, kThreads, 0, stream>>>(ws.logits, ws.partials, int(ws.n_chunks), L,
                                                            logscore, rows_per_cta);

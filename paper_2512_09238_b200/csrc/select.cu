@@ -1,7 +1,8 @@
 // tca_select: core-context selection of Eqs. 6-8 (Algorithm 2, lines 2-6).
 //
 //   block_metric_kernel  one warp per block: h_j of Eq. 6 from log s, in fp64
-//   block_rank_kernel    rank of every block in ascending (h, index) order by counting,
+//   block_rank_kernel    rank of every block in ascending (h, index) order by counting
+//                        (8 threads per block over shared-memory tiles of keys),
 //                        then t_j = Psi[rank_j] of Eq. 7
 //   block_topt_kernel    one warp per block: the t_j largest scores by an MSB-first radix
 //                        select on order-preserving 64-bit keys, ties to the lower
@@ -60,29 +61,36 @@ block_metric_kernel(const double* __restrict__ logscore, int64_t L, int m, int b
   }
 }
 
-__global__ void __launch_bounds__(128)
+constexpr int kRankThreads = 256, kRankParts = 8, kRankBlocks = kRankThreads / kRankParts;
+
+// 32 blocks per CTA, 8 threads per block: thread (j, part) counts the keys i = part (mod 8)
+// that sort before block j; the 8 counts are added with shuffles.
+__global__ void __launch_bounds__(kRankThreads)
 block_rank_kernel(const unsigned long long* __restrict__ hkey, int m, int n_kv_heads, int nK,
                   BudgetCounts counts, int32_t* __restrict__ t_ws, int32_t* __restrict__ t_out) {
-  constexpr int kTile = 1024;
+  constexpr int kTile = 2048;
   __shared__ unsigned long long tile[kTile];
   const int u = blockIdx.y;
-  const int j = blockIdx.x * 128 + threadIdx.x;
+  const int part = threadIdx.x & (kRankParts - 1);
+  const int j = blockIdx.x * kRankBlocks + (threadIdx.x >> 3);
   const unsigned long long* hk = hkey + size_t(u) * m;
   const unsigned long long mine = (j < m) ? hk[j] : 0ull;
   int rank = 0;
   for (int i0 = 0; i0 < m; i0 += kTile) {
     const int n = min(kTile, m - i0);
     __syncthreads();
-    for (int i = threadIdx.x; i < n; i += 128) tile[i] = hk[i0 + i];
+    for (int i = threadIdx.x; i < n; i += kRankThreads) tile[i] = hk[i0 + i];
     __syncthreads();
-    if (j < m) {
-      for (int i = 0; i < n; ++i) {
-        unsigned long long other = tile[i];
-        rank += (other < mine) || (other == mine && (i0 + i) < j);
-      }
+#pragma unroll 4
+    for (int i = part; i < n; i += kRankParts) {
+      const unsigned long long other = tile[i];
+      rank += (other < mine) || (other == mine && (i0 + i) < j);
     }
   }
-  if (j >= m) return;
+  rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+  rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+  rank += __shfl_xor_sync(0xffffffffu, rank, 4);
+  if (j >= m || part != 0) return;
   const int h = u % n_kv_heads;
   int t = 1 << (nK - 1);
   for (int k = nK - 1; k >= 0; --k)
@@ -178,7 +186,7 @@ extern "C" int tca_select(const tca_params* prm, const double* logscore, int64_t
       logscore, L, int(m), prm->block, double(prm->alpha), lay.hkey, h_out);
   st = check_launch();
   if (st != TCA_OK) return st;
-  block_rank_kernel<<<dim3(unsigned((m + 127) / 128), unsigned(U)), 128, 0, s>>>(
+  block_rank_kernel<<<dim3(unsigned((m + kRankBlocks - 1) / kRankBlocks), unsigned(U)), kRankThreads, 0, s>>>(
       lay.hkey, int(m), prm->n_kv_heads, nK, counts, lay.t, t_out);
   st = check_launch();
   if (st != TCA_OK) return st;
