@@ -46,6 +46,29 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+# ----------------------------------------------------------------------------- multi-rank plumbing
+def replica_workload(wl, rank: int):
+    """Every rank runs its own replica of the workload on its own batch (seed shifted by rank).
+    The path has no exchange step, so nothing but the timing crosses ranks."""
+    return wl.scaled(seed=wl.seed + 1000 * rank)
+
+
+def reduce_max(values, world: int, device="cpu"):
+    """Element-wise maximum over ranks of a list of floats (a job is as slow as its slowest rank)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_throughput(world: int, batch: int, tokens: int, ms: float) -> float:
+    """Tokens per second of the whole job: every rank processed batch * tokens in `ms`."""
+    return world * batch * tokens / (ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
@@ -310,7 +333,7 @@ def main():
         dist.barrier()
     B.lib()
 
-    wl_rank = wl.scaled(seed=wl.seed + 1000 * rank)        # every replica draws its own batch
+    wl_rank = replica_workload(wl, rank)
     data = I.generate(wl_rank)
     p = I.budget_table(wl)
     pipe = Pipeline(wl_rank, data, p, torch, B, host_io=not args.no_e2e)
@@ -338,18 +361,15 @@ def main():
         clocks = sampler.stop()
         ms = e0.elapsed_time(e1)
         stages = pipe.stage_ms()
-        if world > 1:
-            t = torch.tensor([ms] + [stages[k] for k in sorted(stages)], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t[0])
-            stages = {k: float(v) for k, v in zip(sorted(stages), t[1:])}
+        red = reduce_max([ms] + [stages[k] for k in sorted(stages)], world, device="cuda")
+        ms, stages = red[0], dict(zip(sorted(stages), red[1:]))
         return ms / args.steps, stages, clocks
 
     ms_step, stages, clocks = timed(host_io=False)
     assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
     work = pipe.algorithmic_work()
     prefill_ms = stages["score"] + stages["select"] + stages["compact"] + stages["prefill"]
-    value = world * wl.batch * wl.L / (prefill_ms * 1e-3)
+    value = job_throughput(world, wl.batch, wl.L, prefill_ms)
     decode_us = stages["decode"] * 1e3 / max(1, wl.decode_steps)
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -387,7 +407,7 @@ def main():
         h2d = wl.L * (nQ + 2 * nKV) + wl.decode_steps * (nQ + 2 * nKV)
         d2h = wl.L * nQ + wl.decode_steps * nQ
         e2e_prefill_ms = sum(st_e2e[k] for k in ("h2d", "score", "select", "compact", "prefill", "prefill_io"))
-        out["e2e"] = {"value": world * wl.batch * wl.L / (e2e_prefill_ms * 1e-3), "unit": UNIT,
+        out["e2e"] = {"value": job_throughput(world, wl.batch, wl.L, e2e_prefill_ms), "unit": UNIT,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                       "prefill_ms": e2e_prefill_ms,
                       "decode_us_per_step": st_e2e["decode"] * 1e3 / max(1, wl.decode_steps),

@@ -1,0 +1,198 @@
+"""Parity at the full benchmark sizes, through the same Pipeline object bench.py times.
+
+The oracle cannot afford every output at L = 32K..128K, so selection is checked in full
+(it is O(L)) and attention on sampled rows / sampled decode steps: first and last rows, rows
+around the window, block and tile edges, plus random ones.
+"""
+import numpy as np
+import pytest
+import torch
+
+import bench
+import tca_harness as H
+from oracle import tca_oracle as O
+from paper_2512_09238_b200 import binding as B
+from paper_2512_09238_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _pipeline(wl):
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    return data, p, bench.Pipeline(wl, data, p, torch, B, host_io=False)
+
+
+def _check_selection(wl, data, p, pipe, units):
+    idx = pipe.idx.cpu().numpy()
+    sel = {}
+    accepted = 0
+    for u in units:
+        s, h = divmod(u, wl.n_kv_heads)
+        res = H.oracle_select_unit(wl, data, p, s, h, wl.L)
+        S = idx[pipe.offsets[u]:pipe.offsets[u + 1]].astype(np.int64)
+        t = np.bincount(S // wl.block, minlength=res["m"])
+        accepted += H.compare_selection(res, S, t, wl.block)
+        sel[u] = S
+    assert accepted <= 4
+    return sel
+
+
+def _check_prefill_rows(wl, data, pipe, sel, n_random, heads_per_unit=1):
+    out = pipe.O
+    scale, G = H.scale_of(wl), wl.group
+    m = wl.n_blocks
+    for u, S in sel.items():
+        s, h = divmod(u, wl.n_kv_heads)
+        T = O.retained_set(S, m, wl.block, wl.L)
+        K, V = I.widen(data["k"][s, h, :wl.L]), I.widen(data["v"][s, h, :wl.L])
+        rows = H.sample_rows(wl.L, wl.window, wl.block, n_random, seed=u)
+        for g in range(heads_per_unit):
+            hq = h * G + (g * 3 + u) % G
+            Q = I.widen(data["q"][s, hq, :wl.L])
+            want = O.attention_rows(Q, K, V, T, wl.window, scale, rows)
+            got = H.from_device(out[s, hq][torch.tensor(rows, device="cuda")])
+            H.check_attention(got, want, wl.dtype, f"{wl.name} unit {u} head {hq}")
+
+
+def test_config3_prefill_32k():
+    wl = I.WORKLOADS["config3"]
+    data, p, pipe = _pipeline(wl)
+    pipe.step()
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    sel = _check_selection(wl, data, p, pipe, range(pipe.U))
+    _check_prefill_rows(wl, data, pipe, sel, n_random=10, heads_per_unit=2)
+    # retained-token counts equal each head's budget
+    for u in range(pipe.U):
+        assert len(sel[u]) == pipe.n_sel[u % wl.n_kv_heads] == pipe.cache.n_global[u]
+
+
+def test_config4_prefill_128k_then_256_decode_steps():
+    wl = I.WORKLOADS["config4"]
+    data, p, pipe = _pipeline(wl)
+    B_, prm, L, G = B, pipe.prm, wl.L, wl.group
+    # the step, with the decode loop unrolled here so that chosen steps can be checked
+    pipe.steps_decode = 0
+    pipe.step()
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    units = range(pipe.U)
+    sel = _check_selection(wl, data, p, pipe, units)
+    _check_prefill_rows(wl, data, pipe, {u: sel[u] for u in (0, 3, 5)}, n_random=6)
+    scale = H.scale_of(wl)
+    caches = {u: O.DecodeCache.from_prefill(sel[u], wl.n_blocks, L, wl.block, wl.window, p[u % wl.n_kv_heads], scale)
+              for u in units}
+    Kw = {u: I.widen(data["k"][0, u]) for u in (1, 6)}
+    Vw = {u: I.widen(data["v"][0, u]) for u in (1, 6)}
+    check_steps = {0, 126, 127, 128, 255}
+    for step in range(wl.decode_steps):
+        pos = L + step
+        B_.tca_cache_append(prm, pipe.cache, pipe.kd[step], pipe.vd[step], pipe.qd[step])
+        B_.tca_attn_decode(prm, pipe.qd[step], pipe.cache, pipe.Od[step], pipe.ws_decode)
+        for u in units:
+            Ku = Kw[u] if u in Kw else I.widen(data["k"][0, u, pos - wl.window - wl.block:pos + 1])
+            if u in Kw:
+                caches[u].append(pos, I.widen(data["q"][0, u * G:(u + 1) * G, pos]), Ku)
+            else:   # only the block that may be compressed is needed: index it relative to its start
+                class _Shift:
+                    def __init__(self, a, off): self.a, self.off = a, off
+                    def __getitem__(self, ix): return self.a[np.asarray(ix) - self.off]
+                caches[u].append(pos, I.widen(data["q"][0, u * G:(u + 1) * G, pos]),
+                                 _Shift(Ku, pos - wl.window - wl.block))
+        if step in check_steps:
+            out = H.from_device(pipe.Od[step])
+            for u in (1, 6):
+                for g in (0, G - 1):
+                    want = caches[u].attend(I.widen(data["q"][0, u * G + g, pos]), Kw[u], Vw[u])
+                    H.check_attention(out[0, u * G + g], want, wl.dtype, f"config4 decode step {step}")
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(pipe.ws_decode) == B.TCA_OK
+    cpos = pipe.cache.pos.cpu().numpy()
+    for u in units:
+        np.testing.assert_array_equal(cpos[pipe.cache.unit_rows(u)], caches[u].positions())
+        assert pipe.cache.n_global[u] == len(sel[u]) + 2 * pipe.tbar[u % wl.n_kv_heads]   # two blocks compressed
+
+
+def test_config2_decode_32k_batch4_and_dense_decode():
+    wl = I.WORKLOADS["config2"]
+    data, p, pipe = _pipeline(wl)
+    L, G = wl.L, wl.group
+    # setup (score with the newest query, select, compact), then the timed call: one decode step
+    B.tca_score(pipe.prm, pipe.q_last, pipe.Kp, L, pipe.logscore, pipe.ws_score)
+    B.tca_select(pipe.prm, pipe.logscore, L, pipe.n_k, pipe.idx, pipe.offsets_dev, None, None, pipe.ws_select)
+    B.tca_compact_kv(pipe.prm, pipe.Kp, pipe.Vp, L, pipe.idx, pipe.offsets_dev, pipe.offsets, pipe.cache)
+    out = torch.empty_like(pipe.q_last)
+    B.tca_attn_decode(pipe.prm, pipe.q_last, pipe.cache, out, pipe.ws_decode)
+    torch.cuda.synchronize()
+    units = [0, 7, 13, 22, 31]
+    sel = _check_selection(wl, data, p, pipe, units)
+    got = H.from_device(out)
+    scale = H.scale_of(wl)
+    for u in units:
+        s, h = divmod(u, wl.n_kv_heads)
+        T = O.retained_set(sel[u], wl.n_blocks, wl.block, L)
+        K, V = I.widen(data["k"][s, h, :L]), I.widen(data["v"][s, h, :L])
+        for g in range(G):
+            want = O.attention_over_set(I.widen(data["q"][s, h * G + g, L - 1]), K[T], V[T], scale)
+            H.check_attention(got[s, h * G + g], want, wl.dtype, f"config2 decode unit {u}")
+    # dense decode over the full cache (100 % budget) against plain softmax attention
+    dense = wl.scaled(budget=("fixed", 1.0))
+    pd = I.budget_table(dense)
+    pipe_d = bench.Pipeline(dense, data, pd, torch, B, host_io=False)
+    B.tca_score(pipe_d.prm, pipe_d.q_last, pipe_d.Kp, L, pipe_d.logscore, pipe_d.ws_score)
+    B.tca_select(pipe_d.prm, pipe_d.logscore, L, pipe_d.n_k, pipe_d.idx, pipe_d.offsets_dev, None, None,
+                 pipe_d.ws_select)
+    B.tca_compact_kv(pipe_d.prm, pipe_d.Kp, pipe_d.Vp, L, pipe_d.idx, pipe_d.offsets_dev, pipe_d.offsets,
+                     pipe_d.cache)
+    B.tca_attn_decode(pipe_d.prm, pipe_d.q_last, pipe_d.cache, out, pipe_d.ws_decode)
+    torch.cuda.synchronize()
+    assert int(pipe_d.cache.n_global.sum() + pipe_d.cache.n_tail.sum()) == pipe_d.U * L
+    got = H.from_device(out)
+    for u in (0, 31):
+        s, h = divmod(u, wl.n_kv_heads)
+        K, V = I.widen(data["k"][s, h, :L]), I.widen(data["v"][s, h, :L])
+        for g in (0, 3):
+            q = I.widen(data["q"][s, h * G + g, L - 1])
+            x = (K @ q) * scale
+            w = np.exp(x - x.max())
+            H.check_attention(got[s, h * G + g], (w / w.sum()) @ V, wl.dtype, "config2 dense decode")
+
+
+@pytest.mark.parametrize("frac", [0.05, 0.10, 0.25, 0.50, 1.0])
+def test_config5_budget_sweep_64k(frac):
+    wl = I.WORKLOADS["config5"].scaled(budget=("fixed", frac))
+    data, p, pipe = _pipeline(wl)
+    pipe.step()
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    units = [0, 5, 11, 15]
+    sel = _check_selection(wl, data, p, pipe, units)
+    m = wl.n_blocks
+    for u in units:   # uniform budget: every head keeps the same count, and sees it in its cache
+        assert len(sel[u]) == pipe.n_sel[0]
+        assert abs(len(sel[u]) / (m * wl.block) - frac) < 0.01
+    _check_prefill_rows(wl, data, pipe, {u: sel[u] for u in units[:2]}, n_random=4)
+    if frac == 1.0:   # the library's own dense baseline really is dense causal attention
+        u = 11
+        s, h = divmod(u, wl.n_kv_heads)
+        np.testing.assert_array_equal(sel[u], np.arange(m * wl.block))
+        K, V = I.widen(data["k"][s, h, :wl.L]), I.widen(data["v"][s, h, :wl.L])
+        Q = I.widen(data["q"][s, h * wl.group + 1, :wl.L])
+        for i in (0, 4095, 4096, 40000, wl.L - 1):
+            x = (K[:i + 1] @ Q[i]) * H.scale_of(wl)
+            w = np.exp(x - x.max())
+            H.check_attention(H.from_device(pipe.O[s, h * wl.group + 1, i]), (w / w.sum()) @ V[:i + 1], wl.dtype,
+                              f"dense row {i}")
+    # the 64 decode steps ran inside step(): compare the last one with the oracle replaying the appends
+    scale, G, L = H.scale_of(wl), wl.group, wl.L
+    u = units[1]
+    s, h = divmod(u, wl.n_kv_heads)
+    cache = O.DecodeCache.from_prefill(sel[u], m, L, wl.block, wl.window, p[h], scale)
+    Kw, Vw = I.widen(data["k"][s, h]), I.widen(data["v"][s, h])
+    for step in range(wl.decode_steps):
+        kept = cache.append(L + step, I.widen(data["q"][s, h * G:(h + 1) * G, L + step]), Kw)
+        assert kept is None          # 64 steps never complete a block of 128
+    last = wl.decode_steps - 1
+    want = cache.attend(I.widen(data["q"][s, h * G + 2, L + last]), Kw, Vw)
+    H.check_attention(H.from_device(pipe.Od[last, s, h * G + 2]), want, wl.dtype, f"config5 decode f={frac}")
