@@ -283,6 +283,7 @@ def main():
     ap.add_argument("--length", type=int, default=0, help="override L (smaller runs for profiling)")
     ap.add_argument("--decode-steps", type=int, default=-1)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-dense", action="store_true", help="skip the 100 %-budget comparison run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
 
@@ -398,6 +399,22 @@ def main():
         "retained_fraction": work["retained_fraction"],
         "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
     }
+
+    if not args.no_dense:
+        # this library's own dense path: the same calls with a 100 % budget (p_b = 1 for every head)
+        dense_wl = wl_rank.scaled(budget=("fixed", 1.0))
+        main_pipe = pipe
+        pipe = Pipeline(dense_wl, data, I.budget_table(dense_wl), torch, B, host_io=False)
+        _, st_dense, _ = timed(host_io=False)
+        dense_prefill = st_dense["score"] + st_dense["select"] + st_dense["compact"] + st_dense["prefill"]
+        dense_decode_us = st_dense["decode"] * 1e3 / max(1, wl.decode_steps)
+        out["dense_baseline"] = {"budget": 1.0, "prefill_ms": dense_prefill, "decode_us_per_step": dense_decode_us,
+                                 "speedup_prefill": dense_prefill / prefill_ms,
+                                 "speedup_decode": dense_decode_us / decode_us if decode_us > 0 else None,
+                                 "kv_rows_retained_vs_dense": work["retained_fraction"]}
+        del pipe
+        torch.cuda.empty_cache()
+        pipe = main_pipe
 
     if not args.no_e2e:
         ms_e2e, st_e2e, _ = timed(host_io=True)

@@ -237,24 +237,26 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
           ok = ptx::mbar_wait(&bars[BAR_S + h], uint32_t(t) & 1u, abort_flag);
           if (!ok) break;
           ptx::tc_fence_after();
-          // pass 1: row maximum
-          float mx = -INFINITY;
-#pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
-            uint32_t v[32];
-            ptx::tmem_ld32(lane_addr + Cfg::colS(h) + c * 32, v);
-            ptx::tc_wait_ld();
-            if (masked) {
+          // the whole row of S (128 fp32) into registers with one wait
+          uint32_t v[BN];
 #pragma unroll
-              for (int k = 0; k < 32; ++k) {
-                const int col = c * 32 + k;
-                if (col >= lo && col <= hi) mx = fmaxf(mx, __uint_as_float(v[k]));
-              }
-            } else {
+          for (int c = 0; c < BN / 32; ++c)
+            ptx::tmem_ld32(lane_addr + Cfg::colS(h) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+          ptx::tc_wait_ld();
+          if (masked) {   // a masked score is -inf: it loses every max and its exponential is exactly 0
 #pragma unroll
-              for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(v[k]));
-            }
+            for (int k = 0; k < BN; ++k)
+              if (k < lo || k > hi) v[k] = 0xff800000u;
           }
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int k = 0; k < BN; k += 4) {
+            mx4[0] = fmaxf(mx4[0], __uint_as_float(v[k]));
+            mx4[1] = fmaxf(mx4[1], __uint_as_float(v[k + 1]));
+            mx4[2] = fmaxf(mx4[2], __uint_as_float(v[k + 2]));
+            mx4[3] = fmaxf(mx4[3], __uint_as_float(v[k + 3]));
+          }
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           m_run = fmaxf(m_run, mx * scale_log2e);
           // lazy rescale of the accumulator (warp-uniform decision: TMEM access is warp-wide)
           if (__any_sync(0xffffffffu, m_run > m_used + kRescaleThreshold)) {
@@ -262,47 +264,37 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
             if (t > 0) {
 #pragma unroll 1
               for (int c = 0; c < D / 32; ++c) {
-                uint32_t v[32];
-                ptx::tmem_ld32(lane_addr + Cfg::colO(h) + c * 32, v);
+                uint32_t o[32];
+                ptx::tmem_ld32(lane_addr + Cfg::colO(h) + c * 32, o);
                 ptx::tc_wait_ld();
 #pragma unroll
-                for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * alpha);
-                ptx::tmem_st32(lane_addr + Cfg::colO(h) + c * 32, v);
+                for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                ptx::tmem_st32(lane_addr + Cfg::colO(h) + c * 32, o);
               }
               ptx::tc_wait_st();
             }
             l *= alpha;
             m_used = m_run;
           }
-          // pass 2: p = exp2(s*scale - m), row sum, bf16 P into swizzled shared memory
-          const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
-          float sum = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
-            uint32_t v[32];
-            ptx::tmem_ld32(lane_addr + Cfg::colS(h) + c * 32, v);
-            ptx::tc_wait_ld();
-            float p[32];
+          // p = exp2(s*scale - m), row sum, bf16 P into swizzled shared memory
+          const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+          float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-              const int col = c * 32 + k;
-              float e = ptx::fast_exp2(fmaf(__uint_as_float(v[k]), scale_log2e, -m_sub));
-              if (masked && (col < lo || col > hi)) e = 0.f;
-              p[k] = e;
-              sum += e;
-            }
-            uint8_t* dst = p_row + (c >> 1) * kHalfBytes;
+          for (int q = 0; q < BN / 8; ++q) {
+            float e[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint4 w;
-              w.x = ptx::pack_bf16x2(p[q * 8 + 0], p[q * 8 + 1]);
-              w.y = ptx::pack_bf16x2(p[q * 8 + 2], p[q * 8 + 3]);
-              w.z = ptx::pack_bf16x2(p[q * 8 + 4], p[q * 8 + 5]);
-              w.w = ptx::pack_bf16x2(p[q * 8 + 6], p[q * 8 + 7]);
-              const int chunk = (c & 1) * 4 + q;
-              *reinterpret_cast<uint4*>(dst + ((chunk ^ (row & 7)) << 4)) = w;
+            for (int k = 0; k < 8; ++k) {
+              e[k] = ptx::fast_exp2(fmaf(__uint_as_float(v[q * 8 + k]), scale_log2e, neg_m));
+              sum4[k & 3] += e[k];
             }
+            uint4 w;
+            w.x = ptx::pack_bf16x2(e[0], e[1]);
+            w.y = ptx::pack_bf16x2(e[2], e[3]);
+            w.z = ptx::pack_bf16x2(e[4], e[5]);
+            w.w = ptx::pack_bf16x2(e[6], e[7]);
+            *reinterpret_cast<uint4*>(p_row + (q >> 3) * kHalfBytes + (((q & 7) ^ (row & 7)) << 4)) = w;
           }
+          const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
           l += sum;
           ptx::fence_proxy_async_smem();
           ptx::tc_fence_before();
