@@ -15,7 +15,8 @@
 //
 // Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-5 /
 // 6-9 = softmax of head 0 / head 1 (one thread per query row = one TMEM lane).
-// TMEM (512 columns): S0 | S1 | O0 | O1.  Shared memory: Q0 Q1 | 3-slot K/V ring | P0 P1.
+// TMEM (512 columns): S0 | S1 | O0 | O1; the bf16 P of a tile overwrites the first half of its
+// S columns and feeds the PV product straight from TMEM.  Shared memory: Q0 Q1 | 5-slot K/V ring.
 // Per tile the issuer runs  PV0(t) S0(t+1) PV1(t) S1(t+1)  so that S of one head is being
 // computed while the other head's softmax is in flight.  O stays in TMEM and is rescaled
 // lazily: only when a row maximum grew by more than 2^8 since the last rescale.
@@ -34,7 +35,7 @@ namespace {
 
 constexpr int BM = 128, BN = 128;
 constexpr int kThreads = 320;
-constexpr int kRing = 3;
+constexpr int kRing = 5;
 constexpr int kHalfBytes = 128 * 128;  // 128 rows x 128 bytes (64 bf16): one swizzled box
 constexpr float kRescaleThreshold = 8.f;
 
@@ -43,17 +44,17 @@ struct TcCfg {
   static constexpr int NH = D / 64;                 // 64-element halves per row
   static constexpr int kQ = NH * kHalfBytes;        // one head's Q tile
   static constexpr int kKV = NH * kHalfBytes;       // one K or V tile
-  static constexpr int kP = 2 * kHalfBytes;         // 128 x 128 bf16
   static constexpr int offQ = 0;
   static constexpr int offKV = 2 * kQ;
-  static constexpr int offP = offKV + kRing * kKV;
-  static constexpr int offBar = offP + 2 * kP;
+  static constexpr int offBar = offKV + kRing * kKV;
   static constexpr int bytes = offBar + 256 + 1024;  // + barriers/scalars + alignment slack
+  static constexpr uint32_t colP(int h) { return uint32_t(h) * 128u; }   // bf16 P overwrites the first half of S
   static constexpr uint32_t colS(int h) { return uint32_t(h) * 128u; }
   static constexpr uint32_t colO(int h) { return 256u + uint32_t(h) * uint32_t(D); }
 };
 
-enum { BAR_Q = 0, BAR_FULL = 1, BAR_EMPTY = 4, BAR_S = 7, BAR_P = 9, BAR_PV = 11, N_BARS = 13 };
+enum { BAR_Q = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + kRing, BAR_S = BAR_EMPTY + kRing, BAR_P = BAR_S + 2,
+       BAR_PV = BAR_P + 2, N_BARS = BAR_PV + 2 };
 
 struct TileGeom {
   int n_gt, nt;
@@ -83,7 +84,8 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::offBar);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  static_assert(N_BARS <= 24, "barrier block");
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* s_nvis = reinterpret_cast<int*>(tmem_slot + 2);
 
@@ -163,24 +165,30 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         constexpr uint32_t idescPV = ptx::idesc_bf16(BM, D, true);
         const uint32_t q_base = ptx::smem_u32(smem + Cfg::offQ);
         const uint32_t kv_base = ptx::smem_u32(smem + Cfg::offKV);
-        const uint32_t p_base = ptx::smem_u32(smem + Cfg::offP);
+        // Descriptors differ only in their 14-bit start-address field (bytes >> 4) and every
+        // operand lives below 256 KB, so a k-step or a ring slot is one add on the low word.
+        const uint64_t dq = ptx::smem_desc_sw128(q_base, 16, 1024);
+        const uint64_t dk = ptx::smem_desc_sw128(kv_base, 16, 1024);           // K tile as K-major B
+        const uint64_t dv = ptx::smem_desc_sw128(kv_base, kHalfBytes, 1024);   // V tile as MN-major B
         auto issue_S = [&](int h, int slot) {
+          const uint64_t a0 = dq + uint64_t(uint32_t(h * Cfg::kQ) >> 4);
+          const uint64_t b0 = dk + uint64_t(uint32_t(slot * Cfg::kKV) >> 4);
+          const uint32_t d = tmem_base + Cfg::colS(h);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = uint32_t(kk >> 2) * kHalfBytes + uint32_t(kk & 3) * 32u;
-            const uint64_t a = ptx::smem_desc_sw128(q_base + h * Cfg::kQ + off, 16, 1024);
-            const uint64_t b = ptx::smem_desc_sw128(kv_base + slot * Cfg::kKV + off, 16, 1024);
-            ptx::umma_ss(tmem_base + Cfg::colS(h), a, b, idescS, kk > 0);
+            const uint32_t off = (uint32_t(kk >> 2) * kHalfBytes + uint32_t(kk & 3) * 32u) >> 4;
+            ptx::umma_ss(d, a0 + off, b0 + off, idescS, kk > 0);
           }
         };
+        // O += P V with P read from TMEM (it overwrote the first 64 columns of S as packed bf16):
+        // the A operand costs no shared-memory bandwidth.
         auto issue_PV = [&](int h, int slot, bool acc) {
+          const uint64_t b0 = dv + uint64_t(uint32_t(slot * Cfg::kKV) >> 4);
+          const uint32_t d = tmem_base + Cfg::colO(h);
+          const uint32_t a = tmem_base + Cfg::colP(h);
 #pragma unroll
-          for (int kk = 0; kk < BN / 16; ++kk) {
-            const uint32_t offp = uint32_t(kk >> 2) * kHalfBytes + uint32_t(kk & 3) * 32u;
-            const uint64_t a = ptx::smem_desc_sw128(p_base + h * Cfg::kP + offp, 16, 1024);
-            const uint64_t b = ptx::smem_desc_sw128(kv_base + slot * Cfg::kKV + uint32_t(kk) * 2048u, kHalfBytes, 1024);
-            ptx::umma_ss(tmem_base + Cfg::colO(h), a, b, idescPV, (acc || kk > 0) ? 1u : 0u);
-          }
+          for (int kk = 0; kk < BN / 16; ++kk)
+            ptx::umma_ts(d, a + uint32_t(kk * 8), b0 + uint32_t((kk * 2048) >> 4), idescPV, (acc || kk > 0) ? 1u : 0u);
         };
         bool ok = ptx::mbar_wait(&bars[BAR_Q], 0, abort_flag) && ptx::mbar_wait(&bars[BAR_FULL + 0], 0, abort_flag);
         if (ok) {
@@ -222,7 +230,6 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         const int64_t c_i = min(max(int64_t(0), i - window + 1), mb);
         const int nvis_i = lower_bound_pos(pos + seg, n_global, c_i);
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
-        uint8_t* p_row = smem + Cfg::offP + h * Cfg::kP + row * 128;
         float m_run = -INFINITY, m_used = -INFINITY, l = 0.f;
         bool ok = true;
         for (int t = 0; t < nt; ++t) {
@@ -276,7 +283,7 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
             l *= alpha;
             m_used = m_run;
           }
-          // p = exp2(s*scale - m), row sum, bf16 P into swizzled shared memory
+          // p = exp2(s*scale - m), row sum, packed bf16 P back into TMEM over the S columns
           const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
           float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -287,16 +294,18 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
               e[k] = ptx::fast_exp2(fmaf(__uint_as_float(v[q * 8 + k]), scale_log2e, neg_m));
               sum4[k & 3] += e[k];
             }
-            uint4 w;
-            w.x = ptx::pack_bf16x2(e[0], e[1]);
-            w.y = ptx::pack_bf16x2(e[2], e[3]);
-            w.z = ptx::pack_bf16x2(e[4], e[5]);
-            w.w = ptx::pack_bf16x2(e[6], e[7]);
-            *reinterpret_cast<uint4*>(p_row + (q >> 3) * kHalfBytes + (((q & 7) ^ (row & 7)) << 4)) = w;
+            // packed P goes back into v[]: entry q*4+j is never read again (j < 4 <= 8)
+            v[q * 4 + 0] = ptx::pack_bf16x2(e[0], e[1]);
+            v[q * 4 + 1] = ptx::pack_bf16x2(e[2], e[3]);
+            v[q * 4 + 2] = ptx::pack_bf16x2(e[4], e[5]);
+            v[q * 4 + 3] = ptx::pack_bf16x2(e[6], e[7]);
           }
+#pragma unroll
+          for (int c = 0; c < BN / 64; ++c)
+            ptx::tmem_st32(lane_addr + Cfg::colP(h) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+          ptx::tc_wait_st();
           const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
           l += sum;
-          ptx::fence_proxy_async_smem();
           ptx::tc_fence_before();
           ptx::mbar_arrive(&bars[BAR_P + h]);
         }
