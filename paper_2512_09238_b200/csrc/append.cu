@@ -18,6 +18,8 @@ cache_append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, co
                     T* __restrict__ Kc, T* __restrict__ Vc, int32_t* __restrict__ pos,
                     int64_t* __restrict__ state, int64_t tail_cap, int D, int G, int b, int window,
                     double sm_scale) {
+  pdl_wait();                 // the previous step's kernels still read the cache and its state
+  pdl_launch_dependents();
   const int u = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, lane16 = tid & 15, grp = tid >> 4;
   int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
@@ -152,18 +154,17 @@ extern "C" int tca_cache_append(const tca_params* prm, tca_cache_desc* c, const 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (prm->dtype == TCA_BF16) {
     using T = __nv_bfloat16;
-    cache_append_kernel<T><<<unsigned(U), kThreads, 0, s>>>(
-        static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<const T*>(q_cur),
-        static_cast<T*>(c->k), static_cast<T*>(c->v), c->pos, c->state, c->tail_cap, prm->head_dim, G,
-        prm->block, prm->window, double(prm->sm_scale));
+    st = launch_pdl(cache_append_kernel<T>, dim3(unsigned(U)), dim3(kThreads), size_t(0), s,
+                    static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<const T*>(q_cur),
+                    static_cast<T*>(c->k), static_cast<T*>(c->v), c->pos, c->state, c->tail_cap, prm->head_dim, G,
+                    prm->block, prm->window, double(prm->sm_scale));
   } else {
     using T = float;
-    cache_append_kernel<T><<<unsigned(U), kThreads, 0, s>>>(
-        static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<const T*>(q_cur),
-        static_cast<T*>(c->k), static_cast<T*>(c->v), c->pos, c->state, c->tail_cap, prm->head_dim, G,
-        prm->block, prm->window, double(prm->sm_scale));
+    st = launch_pdl(cache_append_kernel<T>, dim3(unsigned(U)), dim3(kThreads), size_t(0), s,
+                    static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<const T*>(q_cur),
+                    static_cast<T*>(c->k), static_cast<T*>(c->v), c->pos, c->state, c->tail_cap, prm->head_dim, G,
+                    prm->block, prm->window, double(prm->sm_scale));
   }
-  st = check_launch();
   if (st != TCA_OK) return st;
   for (int64_t u = 0; u < U; ++u) {
     c->n_tail[u] += 1;

@@ -76,6 +76,27 @@ DecodeWs decode_ws_layout(const tca_params* prm, int64_t rows_total, int64_t n_u
 // ------------------------------------------------------------------ device helpers
 #ifdef __CUDACC__
 
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while its
+// predecessor in the stream is still draining; pdl_wait() blocks until the predecessor has
+// completed and its writes are visible, so it must come before the first dependent access.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <typename... KArgs, typename... Args>
+inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess ? TCA_OK : TCA_ERR_CUDA;
+}
+
 template <typename T>
 struct Elt;
 template <>

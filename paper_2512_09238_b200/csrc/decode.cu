@@ -59,6 +59,8 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
   constexpr int EPL = D / 16;
   constexpr int R = Cfg::R, NB = Cfg::NB;
   constexpr int kStages = Ring::kStages;
+  pdl_wait();
+  pdl_launch_dependents();
   const int u = blockIdx.y;
   const int part_idx = blockIdx.x;
   const UnitView uv = load_unit(state, u, tail_cap);
@@ -285,6 +287,8 @@ __global__ void __launch_bounds__(kThreads)
 decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restrict__ state, int64_t tail_cap,
                       int target, T* __restrict__ O) {
   constexpr int NW = kConsumers / 32;   // warp w merges partials w, w + NW, ...; a lane owns 4 outputs
+  pdl_wait();                 // the partials come from the split kernel
+  pdl_launch_dependents();
   const int g = blockIdx.x, u = blockIdx.y;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int n_chunks = n_parts(uv.len(), target);
@@ -382,9 +386,9 @@ int launch_decode(const tca_params* prm, const void* q, const tca_cache_desc* c,
     st = check_launch();
   }
   if (st != TCA_OK) return st;
-  decode_combine_kernel<T, D, G><<<dim3(G, unsigned(U)), kThreads, 0, stream>>>(ws.partial, c->state, c->tail_cap,
-                                                                               target, static_cast<T*>(O));
-  return check_launch();
+  return launch_pdl(decode_combine_kernel<T, D, G>, dim3(G, unsigned(U)), dim3(kThreads), size_t(0), stream,
+                    static_cast<const float*>(ws.partial), static_cast<const int64_t*>(c->state), c->tail_cap, target,
+                    static_cast<T*>(O));
 }
 
 template <typename T, int D>

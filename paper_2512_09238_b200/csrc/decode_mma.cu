@@ -74,6 +74,8 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   constexpr int kStages = Ring::kStages;
   constexpr int ND = D / 8;     // n8 tiles across the head dimension
   constexpr int KC = D / 16;    // k16 chunks across the head dimension
+  pdl_wait();                 // the cache state and rows come from the kernels before this one
+  pdl_launch_dependents();
   const int u = blockIdx.y, part_idx = blockIdx.x;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int64_t len = uv.len();
@@ -311,10 +313,9 @@ int launch_decode_mma(const tca_params* prm, const void* q, const tca_cache_desc
   auto kern = decode_mma_kernel<D>;
   TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Ring::kSmemBytes));
   dim3 grid(unsigned((max_len + target - 1) / target), unsigned(U));
-  kern<<<grid, kMmaThreads, Ring::kSmemBytes, stream>>>(mk, mv, static_cast<const __nv_bfloat16*>(q), c->state,
-                                                        c->tail_cap, G, prm->sm_scale * 1.4426950408889634f, target,
-                                                        ws.partial, ws.status);
-  return check_launch();
+  return launch_pdl(kern, grid, dim3(kMmaThreads), size_t(Ring::kSmemBytes), stream, mk, mv,
+                    static_cast<const __nv_bfloat16*>(q), static_cast<const int64_t*>(c->state), c->tail_cap, G,
+                    prm->sm_scale * 1.4426950408889634f, target, ws.partial, ws.status);
 }
 
 template int launch_decode_mma<64>(const tca_params*, const void*, const tca_cache_desc*, const DecodeWs&, int64_t,
