@@ -1,10 +1,11 @@
 // tca_score: token importance of Eq. 5 in the log domain.
 //
-// Pass 1 (score_logits_kernel) streams K once with 128-bit loads, 16 lanes per key row,
-// accumulates the G dot products of a query group in fp64 (products of bf16 or fp32
-// inputs are exact in fp64, so the logits are exact up to summation rounding), reduces
-// across lanes with a transposing warp-shuffle butterfly (one exchange per output
-// instead of four), writes the logits and a per-CTA (max, sum-exp) partial per head.
+// Pass 1 (score_logits_kernel) streams K once with 128-bit loads and accumulates the G dot
+// products of a query group in fp64 (products of bf16 or fp32 inputs are exact in fp64, so
+// the logits are exact up to summation rounding: log-scores reach +-50, where fp32 has a
+// 4e-6 ulp against the 1e-5 selection rule).  Four lanes share four key rows (4 x 4 register
+// blocking, queries from shared memory), see the kernel.  Each CTA also leaves a
+// (max, sum-exp) partial per head.
 // Pass 2 (score_finalize_kernel) merges the partials into each head's log-sum-exp and
 // turns logits into  log( (1/G) * sum_g softmax_g[j] ).
 #include "common.cuh"
@@ -13,62 +14,6 @@ namespace tca {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kGroups = kThreads / 16;  // 16-lane groups per CTA, one key row each
-
-template <int G>
-struct ScoreCfg {
-  static constexpr int R = (G == 1) ? 16 : (G == 2) ? 8 : 4;   // rows per lane group per step
-  static constexpr int NV = R * G;                             // values reduced per step
-  static constexpr int NB = (NV + 15) / 16;                    // 16-value butterflies
-  static constexpr int NVP = NB * 16;
-};
-
-// Raw 16-lane row slice: EPL elements per lane.
-template <typename T, int EPL>
-struct RowSlice;
-template <>
-struct RowSlice<__nv_bfloat16, 8> {
-  uint4 raw;
-  __device__ __forceinline__ void load(const __nv_bfloat16* p) { raw = __ldcs(reinterpret_cast<const uint4*>(p)); }
-  __device__ __forceinline__ void zero() { raw = make_uint4(0, 0, 0, 0); }
-  __device__ __forceinline__ double get(int e) const {
-    uint32_t w = (e < 2) ? raw.x : (e < 4) ? raw.y : (e < 6) ? raw.z : raw.w;
-    return (e & 1) ? bf16_hi_to_double(w) : bf16_lo_to_double(w);
-  }
-};
-template <>
-struct RowSlice<__nv_bfloat16, 4> {
-  uint2 raw;
-  __device__ __forceinline__ void load(const __nv_bfloat16* p) { raw = __ldcs(reinterpret_cast<const uint2*>(p)); }
-  __device__ __forceinline__ void zero() { raw = make_uint2(0, 0); }
-  __device__ __forceinline__ double get(int e) const {
-    uint32_t w = (e < 2) ? raw.x : raw.y;
-    return (e & 1) ? bf16_hi_to_double(w) : bf16_lo_to_double(w);
-  }
-};
-template <>
-struct RowSlice<float, 4> {
-  float4 raw;
-  __device__ __forceinline__ void load(const float* p) { raw = __ldcs(reinterpret_cast<const float4*>(p)); }
-  __device__ __forceinline__ void zero() { raw = make_float4(0, 0, 0, 0); }
-  __device__ __forceinline__ double get(int e) const {
-    return double(e == 0 ? raw.x : e == 1 ? raw.y : e == 2 ? raw.z : raw.w);
-  }
-};
-template <>
-struct RowSlice<float, 8> {
-  float4 a, b;
-  __device__ __forceinline__ void load(const float* p) {
-    a = __ldcs(reinterpret_cast<const float4*>(p));
-    b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
-  }
-  __device__ __forceinline__ void zero() { a = b = make_float4(0, 0, 0, 0); }
-  __device__ __forceinline__ double get(int e) const {
-    const float4& v = e < 4 ? a : b;
-    int i = e & 3;
-    return double(i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w);
-  }
-};
 
 __device__ __forceinline__ double elt_to_double(float x) { return double(x); }
 __device__ __forceinline__ double elt_to_double(__nv_bfloat16 x) { return double(__bfloat162float(x)); }
@@ -85,131 +30,138 @@ __device__ __forceinline__ void merge_ml(double& m, double& l, double m2, double
   m = M;
 }
 
-// Transposing butterfly over a 16-lane group: on entry every lane holds 16 partial sums
-// (one per value index), on exit lane i holds the group total of value index i.
-__device__ __forceinline__ double butterfly16(double (&v)[16], int lane16) {
-  {
-    const bool up = lane16 & 8;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      double send = up ? v[i] : v[i + 8];
-      double keep = up ? v[i + 8] : v[i];
-      v[i] = keep + shfl_xor_double(send, 8);
-    }
-  }
-  {
-    const bool up = lane16 & 4;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      double send = up ? v[i] : v[i + 4];
-      double keep = up ? v[i + 4] : v[i];
-      v[i] = keep + shfl_xor_double(send, 4);
-    }
-  }
-  {
-    const bool up = lane16 & 2;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      double send = up ? v[i] : v[i + 2];
-      double keep = up ? v[i + 2] : v[i];
-      v[i] = keep + shfl_xor_double(send, 2);
-    }
-  }
-  {
-    const bool up = lane16 & 1;
-    double send = up ? v[0] : v[1];
-    double keep = up ? v[1] : v[0];
-    v[0] = keep + shfl_xor_double(send, 1);
-  }
-  return v[0];
+// 16-byte chunk -> doubles
+__device__ __forceinline__ void chunk_to_double(const uint4& w, double (&x)[8], __nv_bfloat16) {
+  x[0] = bf16_lo_to_double(w.x); x[1] = bf16_hi_to_double(w.x);
+  x[2] = bf16_lo_to_double(w.y); x[3] = bf16_hi_to_double(w.y);
+  x[4] = bf16_lo_to_double(w.z); x[5] = bf16_hi_to_double(w.z);
+  x[6] = bf16_lo_to_double(w.w); x[7] = bf16_hi_to_double(w.w);
+}
+__device__ __forceinline__ void chunk_to_double(const uint4& w, double (&x)[8], float) {
+  x[0] = double(__uint_as_float(w.x)); x[1] = double(__uint_as_float(w.y));
+  x[2] = double(__uint_as_float(w.z)); x[3] = double(__uint_as_float(w.w));
 }
 
+constexpr int kLogitThreads = 128;
+
+// Register blocking 4 rows x 4 lanes: a group of four lanes owns four consecutive key rows;
+// lane j takes the 16-byte chunks 4i + j of each of them.  A query value fetched from shared
+// memory is then used for four rows (the 128 B/clk return path of shared loads, not the
+// fp64 pipe, limits a one-row-per-thread layout), the sixteen accumulators per lane are
+// independent chains, and the only cross-lane work is a two-step transposing exchange
+// after which lane j holds row j of the group for all G heads.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kLogitThreads)
 score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64_t L, double sm_scale,
                     double* __restrict__ logits, double* __restrict__ partials, int n_chunks) {
-  using Cfg = ScoreCfg<G>;
-  constexpr int EPL = D / 16;
-  constexpr int R = Cfg::R, NB = Cfg::NB;
-  const int u = blockIdx.y;
-  const int chunk = blockIdx.x;
-  const int tid = threadIdx.x;
-  const int lane16 = tid & 15;
-  const int grp = tid >> 4;
+  constexpr int EPC = 16 / int(sizeof(T));          // elements per 16-byte chunk
+  constexpr int kChunks = D / EPC;                  // chunks per row
+  constexpr int kIters = kChunks / 4;               // chunks per lane
+  constexpr int QS = EPC + 2;                       // padded query chunk (doubles): 4 chunks -> 4 bank groups
+  constexpr int kWarps = kLogitThreads / 32;
+  const int u = blockIdx.y, chunk = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int grp = lane >> 2, j = lane & 3;
 
-  // this lane's slice of the G scaled queries
-  double qd[G][EPL];
-  {
-    const T* qu = q_last + (size_t(u) * G) * D + lane16 * EPL;
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) qd[g][e] = elt_to_double(qu[size_t(g) * D + e]) * sm_scale;
+  __shared__ __align__(16) double qs[G][kChunks][QS];
+  __shared__ double red_m[kWarps][G], red_l[kWarps][G];
+  for (int i = tid; i < G * D; i += kLogitThreads) {
+    const int g = i / D, d = i % D;
+    qs[g][d / EPC][d % EPC] = elt_to_double(q_last[(size_t(u) * G) * D + i]) * sm_scale;
   }
+  __syncthreads();
 
-  const T* Ku = K + size_t(u) * L * D + lane16 * EPL;
+  const T* Ku = K + size_t(u) * L * D;
   double* logits_u = logits + size_t(u) * G * L;
   const int64_t row0 = int64_t(chunk) * kScoreChunkRows;
   const int64_t row_end = min(row0 + int64_t(kScoreChunkRows), L);
+  double run_m[G], run_l[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) { run_m[g] = 0.0; run_l[g] = 0.0; }
 
-  double run_m[NB], run_l[NB];
+  for (int64_t base = row0 + warp * 32; base < row_end; base += kWarps * 32) {
+    const int64_t r0 = base + grp * 4;              // the group's four rows
+    double acc[4][G];
 #pragma unroll
-  for (int i = 0; i < NB; ++i) { run_m[i] = 0.0; run_l[i] = 0.0; }
-
-  for (int64_t base = row0; base < row_end; base += kGroups * R) {
-    RowSlice<T, EPL> raw[R];
+    for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-      int64_t row = base + r * kGroups + grp;
-      if (row < row_end) raw[r].load(Ku + size_t(row) * D);
-      else raw[r].zero();
-    }
-    double acc[Cfg::NVP];
+      for (int g = 0; g < G; ++g) acc[rr][g] = 0.0;
 #pragma unroll
-    for (int i = 0; i < Cfg::NVP; ++i) acc[i] = 0.0;
+    for (int i = 0; i < kIters; ++i) {
+      const int c = 4 * i + j;
+      uint4 raw[4];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        double kd = raw[r].get(e);
-#pragma unroll
-        for (int g = 0; g < G; ++g) acc[r * G + g] = fma(qd[g][e], kd, acc[r * G + g]);
+      for (int rr = 0; rr < 4; ++rr) {
+        raw[rr] = make_uint4(0, 0, 0, 0);
+        if (r0 + rr < row_end) raw[rr] = __ldcs(reinterpret_cast<const uint4*>(Ku + size_t(r0 + rr) * D) + c);
       }
 #pragma unroll
-    for (int bf = 0; bf < NB; ++bf) {
-      double part[16];
+      for (int e = 0; e < EPC; e += 2) {
+        double2 qq[G];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) part[i] = acc[bf * 16 + i];
-      double x = butterfly16(part, lane16);
-      int v = bf * 16 + lane16;
-      int r = v / G, g = v - r * G;
-      int64_t row = base + r * kGroups + grp;
-      if (v < Cfg::NV && row < row_end) {
+        for (int g = 0; g < G; ++g) qq[g] = *reinterpret_cast<const double2*>(&qs[g][c][e]);
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) {
+          double x[8];
+          chunk_to_double(raw[rr], x, T());
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            acc[rr][g] = fma(qq[g].x, x[e], acc[rr][g]);
+            acc[rr][g] = fma(qq[g].y, x[e + 1], acc[rr][g]);
+          }
+        }
+      }
+    }
+    // transposing exchange over the four lanes of the group: lane j ends with row j, all heads
+    double half2[2][G];
+    {
+      const bool up = j & 2;
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr)
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const double send = up ? acc[rr][g] : acc[rr + 2][g];
+          const double keep = up ? acc[rr + 2][g] : acc[rr][g];
+          half2[rr][g] = keep + shfl_xor_double(send, 2);
+        }
+    }
+    double xg[G];
+    {
+      const bool up = j & 1;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const double send = up ? half2[0][g] : half2[1][g];
+        const double keep = up ? half2[1][g] : half2[0][g];
+        xg[g] = keep + shfl_xor_double(send, 1);
+      }
+    }
+    const int64_t row = r0 + j;                     // = base + lane: coalesced stores
+    if (row < row_end) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const double x = xg[g];
         logits_u[size_t(g) * L + row] = x;
-        if (run_l[bf] == 0.0) { run_m[bf] = x; run_l[bf] = 1.0; }
-        else if (x > run_m[bf]) { run_l[bf] = run_l[bf] * double(expf(float(run_m[bf] - x))) + 1.0; run_m[bf] = x; }
-        else run_l[bf] += double(expf(float(x - run_m[bf])));
+        if (run_l[g] == 0.0) { run_m[g] = x; run_l[g] = 1.0; }
+        else if (x > run_m[g]) { run_l[g] = run_l[g] * double(expf(float(run_m[g] - x))) + 1.0; run_m[g] = x; }
+        else run_l[g] += double(expf(float(x - run_m[g])));
       }
     }
   }
 
-  // CTA reduction of the per-lane (max, sum-exp): lanes with equal (bf, lane16) share a head.
-  __shared__ double sm_m[NB][kThreads], sm_l[NB][kThreads];
-  __shared__ double cls_m[Cfg::NVP], cls_l[Cfg::NVP];
+  // merge the per-lane (max, sum-exp): lanes by shuffle, warps through shared memory
 #pragma unroll
-  for (int bf = 0; bf < NB; ++bf) { sm_m[bf][tid] = run_m[bf]; sm_l[bf][tid] = run_l[bf]; }
-  __syncthreads();
-  if (tid < Cfg::NVP) {
-    int bf = tid >> 4, l16 = tid & 15;
-    double m = 0.0, l = 0.0;
-    for (int gi = 0; gi < kGroups; ++gi) merge_ml(m, l, sm_m[bf][gi * 16 + l16], sm_l[bf][gi * 16 + l16]);
-    cls_m[tid] = m;
-    cls_l[tid] = l;
+  for (int g = 0; g < G; ++g) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const double m2 = shfl_xor_double(run_m[g], off), l2 = shfl_xor_double(run_l[g], off);
+      merge_ml(run_m[g], run_l[g], m2, l2);
+    }
+    if (lane == 0) { red_m[warp][g] = run_m[g]; red_l[warp][g] = run_l[g]; }
   }
   __syncthreads();
   if (tid < G) {
     double m = 0.0, l = 0.0;
-    for (int v = tid; v < Cfg::NV; v += G) merge_ml(m, l, cls_m[v], cls_l[v]);
+    for (int w = 0; w < kWarps; ++w) merge_ml(m, l, red_m[w][tid], red_l[w][tid]);
     double* p = partials + ((size_t(u) * n_chunks + chunk) * G + tid) * 2;
     p[0] = m;
     p[1] = l;
@@ -269,7 +221,7 @@ int launch_score(const tca_params* prm, const void* q_last, const void* K, int64
                  const ScoreWs& ws, cudaStream_t stream) {
   const int U = prm->batch * prm->n_kv_heads;
   dim3 grid1(unsigned(ws.n_chunks), unsigned(U));
-  score_logits_kernel<T, D, G><<<grid1, kThreads, 0, stream>>>(
+  score_logits_kernel<T, D, G><<<grid1, kLogitThreads, 0, stream>>>(
       static_cast<const T*>(q_last), static_cast<const T*>(K), L, double(prm->sm_scale), ws.logits,
       ws.partials, int(ws.n_chunks));
   int st = check_launch();
