@@ -91,11 +91,13 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = n_q_heads / n_kv_heads;
-  const int U = int(gridDim.x) / (n_qtiles * pairs_per_unit);
-  const int per_tile = U * pairs_per_unit;
-  const int tile = n_qtiles - 1 - int(blockIdx.x) / per_tile;   // long rows first
-  const int rem = int(blockIdx.x) % per_tile;
-  const int u = rem / pairs_per_unit, pair = rem % pairs_per_unit;
+  // Unit-major order: the CTAs resident at any time share one or two KV heads, whose retained
+  // rows and window band then stay in L2; within a unit the long rows go first.
+  const int per_unit = n_qtiles * pairs_per_unit;
+  const int u = int(blockIdx.x) / per_unit;
+  const int rem = int(blockIdx.x) % per_unit;
+  const int tile = n_qtiles - 1 - rem / pairs_per_unit;
+  const int pair = rem % pairs_per_unit;
   const int nh = min(2, G - 2 * pair);                          // heads handled here
   const int seq = u / n_kv_heads, kvh = u % n_kv_heads;
   const int hq0 = seq * n_q_heads + kvh * G + 2 * pair;         // first query head (flattened over batch)
