@@ -19,7 +19,11 @@
 // S columns and feeds the PV product straight from TMEM.  Shared memory: Q0 Q1 | 5-slot K/V ring.
 // Per tile the issuer runs  PV0(t) S0(t+1) PV1(t) S1(t+1)  so that S of one head is being
 // computed while the other head's softmax is in flight.  O stays in TMEM and is rescaled
-// lazily: only when a row maximum grew by more than 2^8 since the last rescale.
+// lazily: only when a row maximum grew by more than 2^8 since the last rescale.  The softmax
+// arithmetic uses the packed fp32x2 forms (fma, add) and the three-input max, which halves its
+// issue slots: the issuer thread shares a warp scheduler with two softmax warps and every slot
+// they take delays the next tcgen05.mma.  CTAs are ordered unit-major so that the CTAs resident
+// at one time read the same one or two KV heads out of L2.
 //
 // Every mbarrier wait is bounded; a wait that gives up raises the status word of the
 // workspace, lets outstanding copies land, frees TMEM and returns.
@@ -38,6 +42,7 @@ constexpr int kThreads = 320;
 constexpr int kRing = 5;
 constexpr int kHalfBytes = 128 * 128;  // 128 rows x 128 bytes (64 bf16): one swizzled box
 constexpr float kRescaleThreshold = 8.f;
+constexpr int kPChunks = 1;   // column chunks in which P is handed to the PV GEMM (2 and 4 measured no faster)
 
 template <int D>
 struct TcCfg {
@@ -54,7 +59,7 @@ struct TcCfg {
 };
 
 enum { BAR_Q = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + kRing, BAR_S = BAR_EMPTY + kRing, BAR_P = BAR_S + 2,
-       BAR_PV = BAR_P + 2, N_BARS = BAR_PV + 2 };
+       BAR_PV = BAR_P + 2 * kPChunks, N_BARS = BAR_PV + 2 };
 
 struct TileGeom {
   int n_gt, nt;
@@ -115,7 +120,7 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
     for (int i = 0; i < kRing; ++i) { ptx::mbar_init(&bars[BAR_FULL + i], 1); ptx::mbar_init(&bars[BAR_EMPTY + i], 1); }
     for (int h = 0; h < 2; ++h) {
       ptx::mbar_init(&bars[BAR_S + h], 1);
-      ptx::mbar_init(&bars[BAR_P + h], 128);
+      for (int c = 0; c < kPChunks; ++c) ptx::mbar_init(&bars[BAR_P + h * kPChunks + c], 128);
       ptx::mbar_init(&bars[BAR_PV + h], 1);
     }
     ptx::fence_barrier_init();
@@ -184,13 +189,24 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         };
         // O += P V with P read from TMEM (it overwrote the first 64 columns of S as packed bf16):
         // the A operand costs no shared-memory bandwidth.
-        auto issue_PV = [&](int h, int slot, bool acc) {
+        // P arrives in kPChunks column chunks, each with its own barrier, so the first k-steps of
+        // PV run while the softmax warps are still exponentiating the rest of the row.
+        auto issue_PV = [&](int h, int slot, bool acc, uint32_t parity) -> bool {
           const uint64_t b0 = dv + uint64_t(uint32_t(slot * Cfg::kKV) >> 4);
           const uint32_t d = tmem_base + Cfg::colO(h);
           const uint32_t a = tmem_base + Cfg::colP(h);
+          constexpr int kPer = BN / 16 / kPChunks;
 #pragma unroll
-          for (int kk = 0; kk < BN / 16; ++kk)
-            ptx::umma_ts(d, a + uint32_t(kk * 8), b0 + uint32_t((kk * 2048) >> 4), idescPV, (acc || kk > 0) ? 1u : 0u);
+          for (int c = 0; c < kPChunks; ++c) {
+            if (!ptx::mbar_wait(&bars[BAR_P + h * kPChunks + c], parity, abort_flag)) return false;
+            ptx::tc_fence_after();
+#pragma unroll
+            for (int k2 = 0; k2 < kPer; ++k2) {
+              const int kk = c * kPer + k2;
+              ptx::umma_ts(d, a + uint32_t(kk * 8), b0 + uint32_t((kk * 2048) >> 4), idescPV, (acc || kk > 0) ? 1u : 0u);
+            }
+          }
+          return true;
         };
         bool ok = ptx::mbar_wait(&bars[BAR_Q], 0, abort_flag) && ptx::mbar_wait(&bars[BAR_FULL + 0], 0, abort_flag);
         if (ok) {
@@ -203,10 +219,8 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
           const int nK = 2 * t + 2, slotK = nK % kRing;
           ok = ptx::mbar_wait(&bars[BAR_FULL + slotV], uint32_t(nV / kRing) & 1u, abort_flag);
           for (int h = 0; h < nh && ok; ++h) {
-            ok = ptx::mbar_wait(&bars[BAR_P + h], uint32_t(t) & 1u, abort_flag);
+            ok = issue_PV(h, slotV, t > 0, uint32_t(t) & 1u);
             if (!ok) break;
-            ptx::tc_fence_after();
-            issue_PV(h, slotV, t > 0);
             ptx::umma_commit(&bars[BAR_PV + h]);
             if (h == nh - 1) ptx::umma_commit(&bars[BAR_EMPTY + slotV]);
             if (t + 1 < nt) {
@@ -259,11 +273,11 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
           }
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (int k = 0; k < BN; k += 4) {
-            mx4[0] = fmaxf(mx4[0], __uint_as_float(v[k]));
-            mx4[1] = fmaxf(mx4[1], __uint_as_float(v[k + 1]));
-            mx4[2] = fmaxf(mx4[2], __uint_as_float(v[k + 2]));
-            mx4[3] = fmaxf(mx4[3], __uint_as_float(v[k + 3]));
+          for (int k = 0; k < BN; k += 8) {
+            mx4[0] = ptx::max3(mx4[0], __uint_as_float(v[k]), __uint_as_float(v[k + 1]));
+            mx4[1] = ptx::max3(mx4[1], __uint_as_float(v[k + 2]), __uint_as_float(v[k + 3]));
+            mx4[2] = ptx::max3(mx4[2], __uint_as_float(v[k + 4]), __uint_as_float(v[k + 5]));
+            mx4[3] = ptx::max3(mx4[3], __uint_as_float(v[k + 6]), __uint_as_float(v[k + 7]));
           }
           const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           m_run = fmaxf(m_run, mx * scale_log2e);
@@ -287,29 +301,33 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
           }
           // p = exp2(s*scale - m), row sum, packed bf16 P back into TMEM over the S columns
           const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-          float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+          const uint64_t scale2 = ptx::pack2(scale_log2e, scale_log2e);
+          const uint64_t neg_m2 = ptx::pack2(neg_m, neg_m);
+          uint64_t sum2[2] = {0ull, 0ull};
+          constexpr int kPairs = BN / 2 / kPChunks;   // packed bf16 words per chunk
 #pragma unroll
-          for (int q = 0; q < BN / 8; ++q) {
-            float e[8];
+          for (int c = 0; c < kPChunks; ++c) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              e[k] = ptx::fast_exp2(fmaf(__uint_as_float(v[q * 8 + k]), scale_log2e, neg_m));
-              sum4[k & 3] += e[k];
+            for (int jj = 0; jj < kPairs; ++jj) {
+              const int j = c * kPairs + jj;
+              float xl, xh;
+              ptx::unpack2(ptx::fma2(ptx::pack2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), scale2, neg_m2),
+                           xl, xh);
+              const float el = ptx::fast_exp2(xl), eh = ptx::fast_exp2(xh);
+              sum2[j & 1] = ptx::add2(sum2[j & 1], ptx::pack2(el, eh));
+              v[j] = ptx::pack_bf16x2(el, eh);   // entry j is never read again (j <= 2j)
             }
-            // packed P goes back into v[]: entry q*4+j is never read again (j < 4 <= 8)
-            v[q * 4 + 0] = ptx::pack_bf16x2(e[0], e[1]);
-            v[q * 4 + 1] = ptx::pack_bf16x2(e[2], e[3]);
-            v[q * 4 + 2] = ptx::pack_bf16x2(e[4], e[5]);
-            v[q * 4 + 3] = ptx::pack_bf16x2(e[6], e[7]);
+            ptx::tmem_st<kPairs>(lane_addr + Cfg::colP(h) + c * kPairs, &v[c * kPairs]);
+            ptx::tc_wait_st();
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(&bars[BAR_P + h * kPChunks + c]);
           }
-#pragma unroll
-          for (int c = 0; c < BN / 64; ++c)
-            ptx::tmem_st32(lane_addr + Cfg::colP(h) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
-          ptx::tc_wait_st();
-          const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-          l += sum;
-          ptx::tc_fence_before();
-          ptx::mbar_arrive(&bars[BAR_P + h]);
+          {
+            float s0, s1, s2, s3;
+            ptx::unpack2(sum2[0], s0, s1);
+            ptx::unpack2(sum2[1], s2, s3);
+            l += (s0 + s1) + (s2 + s3);
+          }
         }
         // epilogue: O / l -> bf16 -> global
         if (ok) ok = ptx::mbar_wait(&bars[BAR_PV + h], uint32_t(nt - 1) & 1u, abort_flag);

@@ -154,6 +154,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+// kWords consecutive 32-bit columns (a multiple of 16) from registers into TMEM.
+template <int kWords>
+__device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t* v) {
+  static_assert(kWords % 16 == 0, "chunk size");
+#pragma unroll
+  for (int i = 0; i < kWords / 32; ++i) tmem_st32(taddr + i * 32, *reinterpret_cast<const uint32_t(*)[32]>(v + i * 32));
+  if constexpr (kWords % 32 != 0) tmem_st16(taddr + (kWords / 32) * 32, v + (kWords / 32) * 32);
+}
+
 // Shared-memory matrix descriptor (128-byte swizzle).  K-major operands: 8-row groups are
 // `sbo` bytes apart, `lbo` is ignored.  MN-major operands: 64-element groups along M/N are
 // `lbo` bytes apart and 8-row groups along K are `sbo` bytes apart.
@@ -182,6 +199,32 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+
+// ------------------------------------------------------------------ packed fp32 pairs (one issue slot for two lanes)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 }  // namespace ptx
