@@ -65,9 +65,10 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
   const int part_idx = blockIdx.x;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int64_t len = uv.len();
-  if (part_idx >= n_parts(len, target)) return;
-  const int64_t row0 = int64_t(part_idx) * target;
-  const int n_rows = int(min(int64_t(target), len - row0));
+  const int np = n_parts(len, target);
+  if (part_idx >= np) return;
+  const int64_t row0 = slice_begin(len, np, part_idx);
+  const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
   const int n_super = (n_rows + kSuperRows - 1) / kSuperRows;
   const int tid = threadIdx.x, lane16 = tid & 15, grp = tid >> 4, warp = tid >> 5;
   const int base_slot = partial_base<kThreads>(state, u, target);
@@ -361,10 +362,24 @@ inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_s
     else
       sms = 148;
   }
-  int64_t target = (total + ctas_per_sm * sms - 1) / (ctas_per_sm * sms);
-  target = (target + kTileRows - 1) / kTileRows * kTileRows;
-  if (target < kSuperRows) target = kSuperRows;
-  return int(target);
+  // Smallest slice length for which the slices of all units fit the resident CTAs in one
+  // wave: with one slice more than that, the extra CTA starts only after another one ends.
+  const int64_t slots = int64_t(ctas_per_sm) * sms;
+  auto count = [&](int64_t target) {
+    int64_t n = 0;
+    for (int64_t u = 0; u < U; ++u) n += (c->n_global[u] + c->n_tail[u] + target - 1) / target;
+    return n;
+  };
+  int64_t lo = (total + slots - 1) / slots, hi = max_len;
+  if (lo < kSuperRows) lo = kSuperRows;
+  if (hi < lo) hi = lo;
+  if (count(lo) > slots) {
+    while (lo < hi) {               // count() does not increase with target
+      const int64_t mid = lo + (hi - lo) / 2;
+      if (count(mid) <= slots) hi = mid; else lo = mid + 1;
+    }
+  }
+  return int(lo);
 }
 
 template <typename T, int D, int G>

@@ -36,8 +36,11 @@ __device__ __forceinline__ UnitView load_unit(const int64_t* state, int u, int64
   return v;
 }
 
-// CTAs of unit u: ceil(len / target).  Partials are packed unit after unit.
+// CTAs of unit u: ceil(len / target).  Partials are packed unit after unit.  The unit's rows
+// are dealt evenly: slice i covers [i*len/n, (i+1)*len/n), never empty and never longer than
+// target, so no CTA carries a short remainder while the others carry full slices.
 __device__ __forceinline__ int n_parts(int64_t len, int target) { return int((len + target - 1) / target); }
+__device__ __forceinline__ int64_t slice_begin(int64_t len, int n, int i) { return (int64_t(i) * len) / n; }
 
 template <int kBlockThreads>
 __device__ __forceinline__ int partial_base(const int64_t* state, int u, int target) {

@@ -79,9 +79,10 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   const int u = blockIdx.y, part_idx = blockIdx.x;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int64_t len = uv.len();
-  if (part_idx >= n_parts(len, target)) return;
-  const int64_t row0 = int64_t(part_idx) * target;
-  const int n_rows = int(min(int64_t(target), len - row0));
+  const int np = n_parts(len, target);
+  if (part_idx >= np) return;
+  const int64_t row0 = slice_begin(len, np, part_idx);
+  const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int base_slot = partial_base<kMmaThreads>(state, u, target);
 
