@@ -71,7 +71,7 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
   const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
   const int n_super = (n_rows + kSuperRows - 1) / kSuperRows;
   const int tid = threadIdx.x, lane16 = tid & 15, grp = tid >> 4, warp = tid >> 5;
-  const int base_slot = partial_base<kThreads>(state, u, target);
+  const int base_slot = partial_base(state, u, target);
 
   extern __shared__ uint8_t dec_smem_raw[];
   uint8_t* ring_buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dec_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -293,7 +293,7 @@ decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restri
   const int g = blockIdx.x, u = blockIdx.y;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int n_chunks = n_parts(uv.len(), target);
-  const int base_slot = partial_base<kThreads>(state, u, target);
+  const int base_slot = partial_base(state, u, target);
   const int tid = threadIdx.x;
   if (tid >= kConsumers) return;
   const float* base = partial + size_t(base_slot) * G * (D + 2) + size_t(g) * (D + 2);
@@ -302,44 +302,48 @@ decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restri
   __shared__ float s_max[NW];
   __shared__ float s_acc[NW][D], s_l[NW];
 
-  float mx = -INFINITY;
-  for (int c = tid; c < n_chunks; c += kConsumers) mx = fmaxf(mx, base[c * stride + D]);
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-  if (lane == 0) s_max[warp] = mx;
-  consumer_sync(kConsumers);
-  mx = s_max[0];
-#pragma unroll
-  for (int w = 1; w < NW; ++w) mx = fmaxf(mx, s_max[w]);
-
-  // independent loads of up to four partials are in flight per lane
+  // One pass: warp w merges partials w, w + NW, ... with a running maximum (the loads do not
+  // depend on it, so several partials are in flight), then the NW warp states are merged in
+  // warp order.  Every partial holds at least one valid row, so its maximum is finite.
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float l = 0.f;
+  float l = 0.f, m = -INFINITY;
   const bool owns = lane * 4 < D;
 #pragma unroll 4
   for (int c = warp; c < n_chunks; c += NW) {
     const float* p = base + c * stride;
-    const float w = exp2f(p[D] - mx);
-    l = fmaf(p[D + 1], w, l);
+    const float pm = p[D], pl = p[D + 1];
+    float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
     if (owns) {
-      const float2 a = *reinterpret_cast<const float2*>(p + lane * 4);
-      const float2 b = *reinterpret_cast<const float2*>(p + lane * 4 + 2);
-      acc[0] = fmaf(a.x, w, acc[0]);
-      acc[1] = fmaf(a.y, w, acc[1]);
-      acc[2] = fmaf(b.x, w, acc[2]);
-      acc[3] = fmaf(b.y, w, acc[3]);
+      a = *reinterpret_cast<const float2*>(p + lane * 4);
+      b = *reinterpret_cast<const float2*>(p + lane * 4 + 2);
     }
+    const float m_new = fmaxf(m, pm);
+    const float keep = exp2f(m - m_new);        // 0 for the first partial (m = -inf, m_new finite)
+    const float w = exp2f(pm - m_new);
+    l = fmaf(l, keep, pl * w);
+    acc[0] = fmaf(acc[0], keep, a.x * w);
+    acc[1] = fmaf(acc[1], keep, a.y * w);
+    acc[2] = fmaf(acc[2], keep, b.x * w);
+    acc[3] = fmaf(acc[3], keep, b.y * w);
+    m = m_new;
   }
   if (owns) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) s_acc[warp][lane * 4 + i] = acc[i];
   }
-  if (lane == 0) s_l[warp] = l;
+  if (lane == 0) { s_l[warp] = l; s_max[warp] = m; }
   consumer_sync(kConsumers);
   if (tid < D) {
+    float M = s_max[0];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) M = fmaxf(M, s_max[w]);
     float a = 0.f, ls = 0.f;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) { a += s_acc[w][tid]; ls += s_l[w]; }
+    for (int w = 0; w < NW; ++w) {
+      const float wgt = (s_max[w] == -INFINITY) ? 0.f : exp2f(s_max[w] - M);   // a warp without partials
+      a = fmaf(s_acc[w][tid], wgt, a);
+      ls = fmaf(s_l[w], wgt, ls);
+    }
     store_elt(O + (size_t(u) * G + g) * D + tid, n_chunks > 0 ? a / ls : 0.f);
   }
 }

@@ -42,25 +42,17 @@ __device__ __forceinline__ UnitView load_unit(const int64_t* state, int u, int64
 __device__ __forceinline__ int n_parts(int64_t len, int target) { return int((len + target - 1) / target); }
 __device__ __forceinline__ int64_t slice_begin(int64_t len, int n, int i) { return (int64_t(i) * len) / n; }
 
-template <int kBlockThreads>
+// Sum of n_parts over the units before u.  Called by whole warps (all 32 lanes active); every
+// lane returns the total.  It needs no CTA-wide barrier, so a producer warp can skip it.
 __device__ __forceinline__ int partial_base(const int64_t* state, int u, int target) {
-  // sum of n_parts over the units before u (all threads of the CTA call this together)
-  __shared__ int s_base[kBlockThreads / 32];
   int part = 0;
-  for (int v = threadIdx.x; v < u; v += kBlockThreads) {
+  for (int v = int(threadIdx.x & 31u); v < u; v += 32) {
     const int64_t* st = state + size_t(v) * TCA_STATE_WORDS;
     part += n_parts(st[TCA_ST_N_GLOBAL] + st[TCA_ST_N_TAIL], target);
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-  if ((threadIdx.x & 31) == 0) s_base[threadIdx.x >> 5] = part;
-  __syncthreads();
-  int total = 0;
-#pragma unroll
-  for (int w = 0; w < kBlockThreads / 32; ++w) total += s_base[w];
-  __syncthreads();
-  return total;
+  return part;
 }
-
 
 }  // namespace tca

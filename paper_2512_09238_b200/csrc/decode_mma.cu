@@ -74,6 +74,21 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   constexpr int kStages = Ring::kStages;
   constexpr int ND = D / 8;     // n8 tiles across the head dimension
   constexpr int KC = D / 16;    // k16 chunks across the head dimension
+  extern __shared__ uint8_t dmma_smem_raw[];
+  uint8_t* ring_buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dmma_smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ BulkRing<kStages> ring;
+  __shared__ int abort_word;
+  __shared__ float s_m[kMmaConsumers / 32][kMaxGroup], s_l[kMmaConsumers / 32][kMaxGroup];
+  volatile int* abort_flag = &abort_word;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // Set-up that reads nothing the previous kernel wrote runs before the dependency wait.
+  if (tid == 0) {
+    ring.init(kMmaConsumers / 32);
+    abort_word = 0;
+    ptx::tma_prefetch_desc(&map_k);
+    ptx::tma_prefetch_desc(&map_v);
+  }
+  __syncthreads();
   pdl_wait();                 // the cache state and rows come from the kernels before this one
   pdl_launch_dependents();
   const int u = blockIdx.y, part_idx = blockIdx.x;
@@ -83,20 +98,6 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   if (part_idx >= np) return;
   const int64_t row0 = slice_begin(len, np, part_idx);
   const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int base_slot = partial_base<kMmaThreads>(state, u, target);
-
-  extern __shared__ uint8_t dmma_smem_raw[];
-  uint8_t* ring_buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dmma_smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ BulkRing<kStages> ring;
-  __shared__ int abort_word;
-  __shared__ float s_m[kMmaConsumers / 32][kMaxGroup], s_l[kMmaConsumers / 32][kMaxGroup];
-  volatile int* abort_flag = &abort_word;
-  if (tid == 0) {
-    ring.init(kMmaConsumers / 32);
-    abort_word = 0;
-  }
-  __syncthreads();
 
   if (warp == kMmaConsumers / 32) {
     // ------------------------------------------------------------- producer
@@ -119,6 +120,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   }
 
   // --------------------------------------------------------------- consumers
+  const int base_slot = partial_base(state, u, target);
   const int gq = lane >> 2, kq = (lane & 3) * 2;   // accumulator row (query head) and column pair
   // Q as the A operand, one k16 chunk of the head dimension per entry (rows >= G are zero)
   uint32_t qa[KC][2];
