@@ -79,6 +79,18 @@ score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64
 #pragma unroll
   for (int g = 0; g < G; ++g) { run_m[g] = 0.0; run_l[g] = 0.0; }
 
+  // The 16-byte pieces of the next step are requested before the current ones are used, so a
+  // warp always has 64 bytes per lane in flight while its fp64 work runs.
+  auto fetch = [&](int64_t base, int i, uint4 (&dst)[4]) {
+    const int64_t r = base + grp * 4;
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+      dst[rr] = make_uint4(0, 0, 0, 0);
+      if (r + rr < row_end) dst[rr] = __ldcs(reinterpret_cast<const uint4*>(Ku + size_t(r + rr) * D) + (4 * i + j));
+    }
+  };
+  uint4 raw[4];
+  fetch(row0 + warp * 32, 0, raw);
   for (int64_t base = row0 + warp * 32; base < row_end; base += kWarps * 32) {
     const int64_t r0 = base + grp * 4;              // the group's four rows
     double acc[4][G];
@@ -89,12 +101,9 @@ score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64
 #pragma unroll
     for (int i = 0; i < kIters; ++i) {
       const int c = 4 * i + j;
-      uint4 raw[4];
-#pragma unroll
-      for (int rr = 0; rr < 4; ++rr) {
-        raw[rr] = make_uint4(0, 0, 0, 0);
-        if (r0 + rr < row_end) raw[rr] = __ldcs(reinterpret_cast<const uint4*>(Ku + size_t(r0 + rr) * D) + c);
-      }
+      uint4 nxt[4];
+      if (i + 1 < kIters) fetch(base, i + 1, nxt);
+      else fetch(base + kWarps * 32, 0, nxt);
 #pragma unroll
       for (int e = 0; e < EPC; e += 2) {
         double2 qq[G];
@@ -111,6 +120,8 @@ score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64
           }
         }
       }
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) raw[rr] = nxt[rr];
     }
     // transposing exchange over the four lanes of the group: lane j ends with row j, all heads
     double half2[2][G];
