@@ -32,6 +32,7 @@ for _p in (ROOT, os.path.join(ROOT, "tests")):
     if _p not in sys.path:
         sys.path.insert(0, _p)
 
+PREFILL_DRAM_BYTES_CONFIG4 = 2.01e9 + 1.06e9   # measured with ncu, see profiles/launch_list_bench_config4_L131072.md
 METRIC = "128K prefill tok/s"
 UNIT = "tok/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -381,8 +382,11 @@ def main():
 
     tf_peak = peaks["bf16_tflops_sustained"]
     achieved_tf = work["prefill_flops"] / (stages["prefill"] * 1e-3) / 1e12
+    # DRAM bytes of one launch of the prefill kernel (dram__bytes_read.sum + dram__bytes_write.sum), from the
+    # one-pass ncu capture of this very workload summarised under profiles/; other sizes were not captured.
+    traffic = PREFILL_DRAM_BYTES_CONFIG4 if (wl.name == "config4" and wl.L == 131072) else None
     out["roofline"] = {"kernel": "tca_attn_prefill", "bound": "tensor", "achieved": achieved_tf, "peak": tf_peak,
-                       "unit": "TFLOP/s", "frac": achieved_tf / tf_peak, "traffic": None,
+                       "unit": "TFLOP/s", "frac": achieved_tf / tf_peak, "traffic": traffic,
                        "peak_kind": f"bf16 sustained, {peak_kind}", "frac_of_burst": achieved_tf / peaks["bf16_tflops"]}
     hbm = peaks["hbm_gbs"]
 
