@@ -171,6 +171,14 @@ class Pipeline:
             self.h_kd = hk[:, :, wl.L:].permute(2, 0, 1, 3).contiguous().pin_memory()
             self.h_vd = hv[:, :, wl.L:].permute(2, 0, 1, 3).contiguous().pin_memory()
             self.h_O = torch.empty_like(self.h_Qp).pin_memory()
+            self.h_q_last = self.h_Qp[:, :, wl.L - 1].contiguous().pin_memory()
+            self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+            n_ranges = max(1, min(16, wl.L // 4096))
+            step_rows = -(-wl.L // n_ranges)
+            step_rows = -(-step_rows // 128) * 128               # TCA_PREFILL_ROW_ALIGN
+            cuts = list(range(0, wl.L, step_rows)) + [wl.L]
+            self.row_ranges = list(zip(cuts[:-1], cuts[1:]))[::-1]
+            self.ws_rows = [B.alloc_workspace(self.prm, wl.L, B.TCA_OP_PREFILL) for _ in self.row_ranges]
             self.h_Od = torch.empty_like(self.h_qd).pin_memory()
         self.launches_per_step = 2 + 3 + 1 + 1 + wl.decode_steps * 3
         self.ev = {}
@@ -181,13 +189,10 @@ class Pipeline:
         self.ev.setdefault(name, []).append(e)
 
     def step(self, host_io: bool = False, mark: bool = False):
+        if host_io:
+            return self.step_from_host(mark)
         B, prm, L = self.B, self.prm, self.L
         if mark: self._ev("t_begin")
-        if host_io:
-            self.Qp.copy_(self.h_Qp, non_blocking=True)
-            self.Kp.copy_(self.h_Kp, non_blocking=True)
-            self.Vp.copy_(self.h_Vp, non_blocking=True)
-            self.q_last.copy_(self.Qp[:, :, L - 1])
         if mark: self._ev("t0")
         B.tca_score(prm, self.q_last, self.Kp, L, self.logscore, self.ws_score)
         if mark: self._ev("t_score")
@@ -197,17 +202,69 @@ class Pipeline:
         if mark: self._ev("t_compact")
         B.tca_attn_prefill(prm, self.Qp, self.Kp, self.Vp, L, self.cache, self.O, self.ws_prefill)
         if mark: self._ev("t_prefill")
-        if host_io:
-            self.h_O.copy_(self.O, non_blocking=True)
-            self.qd.copy_(self.h_qd, non_blocking=True)
-            self.kd.copy_(self.h_kd, non_blocking=True)
-            self.vd.copy_(self.h_vd, non_blocking=True)
         if mark: self._ev("t_prefill_io")
         for s in range(self.steps_decode):
             B.tca_cache_append(prm, self.cache, self.kd[s], self.vd[s], self.qd[s])
             B.tca_attn_decode(prm, self.qd[s], self.cache, self.Od[s], self.ws_decode)
-        if host_io:
-            self.h_Od.copy_(self.Od, non_blocking=True)
+        if mark: self._ev("t_decode")
+
+    def step_from_host(self, mark: bool = False):
+        """The same step with every input in pinned host memory and every output read back.
+
+        K, V and the newest query go first (score, select and compact need nothing else); Q then
+        arrives in row ranges on a copy stream while tca_attn_prefill_rows works on the ranges
+        already there, and each finished range of O leaves on a third stream.  The last range of
+        rows (the longest) is computed first.
+        """
+        B, prm, L, torch = self.B, self.prm, self.L, self.torch
+        cs = torch.cuda.current_stream()
+        if mark: self._ev("t_begin")
+        start = torch.cuda.Event()
+        start.record(cs)
+        self.s_in.wait_event(start)          # the previous step has finished with these buffers
+        self.s_out.wait_event(start)
+        heads = [(b, h) for b in range(self.wl.batch) for h in range(self.wl.n_q_heads)]
+        ev_q = []
+        with torch.cuda.stream(self.s_in):
+            self.Kp.copy_(self.h_Kp, non_blocking=True)
+            self.q_last.copy_(self.h_q_last, non_blocking=True)
+            ev_k = torch.cuda.Event(); ev_k.record(self.s_in)
+            self.Vp.copy_(self.h_Vp, non_blocking=True)
+            ev_v = torch.cuda.Event(); ev_v.record(self.s_in)
+            for (r0, r1) in self.row_ranges:
+                for (b, h) in heads:
+                    self.Qp[b, h, r0:r1].copy_(self.h_Qp[b, h, r0:r1], non_blocking=True)
+                e = torch.cuda.Event(); e.record(self.s_in)
+                ev_q.append(e)
+            self.qd.copy_(self.h_qd, non_blocking=True)
+            self.kd.copy_(self.h_kd, non_blocking=True)
+            self.vd.copy_(self.h_vd, non_blocking=True)
+            ev_dec = torch.cuda.Event(); ev_dec.record(self.s_in)
+        cs.wait_event(ev_k)
+        if mark: self._ev("t0")
+        B.tca_score(prm, self.q_last, self.Kp, L, self.logscore, self.ws_score)
+        if mark: self._ev("t_score")
+        B.tca_select(prm, self.logscore, L, self.n_k, self.idx, self.offsets_dev, None, None, self.ws_select)
+        if mark: self._ev("t_select")
+        cs.wait_event(ev_v)
+        B.tca_compact_kv(prm, self.Kp, self.Vp, L, self.idx, self.offsets_dev, self.offsets, self.cache)
+        if mark: self._ev("t_compact")
+        for i, (r0, r1) in enumerate(self.row_ranges):
+            cs.wait_event(ev_q[i])
+            B.tca_attn_prefill_rows(prm, self.Qp, self.Kp, self.Vp, L, r0, r1, self.cache, self.O, self.ws_rows[i])
+            done = torch.cuda.Event(); done.record(cs)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(done)
+                for (b, h) in heads:
+                    self.h_O[b, h, r0:r1].copy_(self.O[b, h, r0:r1], non_blocking=True)
+        if mark: self._ev("t_prefill")
+        cs.wait_stream(self.s_out)
+        cs.wait_event(ev_dec)
+        if mark: self._ev("t_prefill_io")
+        for s in range(self.steps_decode):
+            B.tca_cache_append(prm, self.cache, self.kd[s], self.vd[s], self.qd[s])
+            B.tca_attn_decode(prm, self.qd[s], self.cache, self.Od[s], self.ws_decode)
+        self.h_Od.copy_(self.Od, non_blocking=True)
         if mark: self._ev("t_decode")
 
     def stage_ms(self):
@@ -422,18 +479,22 @@ def main():
 
     if not args.no_e2e:
         ms_e2e, st_e2e, _ = timed(host_io=True)
+        assert all(B.tca_ws_status(w) == B.TCA_OK for w in pipe.ws_rows)
         elt = 2 if wl.dtype == "bf16" else 4
         nQ = wl.batch * wl.n_q_heads * wl.head_dim * elt
         nKV = wl.batch * wl.n_kv_heads * wl.head_dim * elt
-        h2d = wl.L * (nQ + 2 * nKV) + wl.decode_steps * (nQ + 2 * nKV)
+        h2d = wl.L * (nQ + 2 * nKV) + nQ + wl.decode_steps * (nQ + 2 * nKV)   # prompt, newest query again, decode tokens
         d2h = wl.L * nQ + wl.decode_steps * nQ
         e2e_prefill_ms = sum(st_e2e[k] for k in ("h2d", "score", "select", "compact", "prefill", "prefill_io"))
         out["e2e"] = {"value": job_throughput(world, wl.batch, wl.L, e2e_prefill_ms), "unit": UNIT,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                       "prefill_ms": e2e_prefill_ms,
                       "decode_us_per_step": st_e2e["decode"] * 1e3 / max(1, wl.decode_steps),
-                      "note": "same calls with pinned host buffers: Q, K, V copied in and O copied back inside "
-                              "the timed prefill; decode tokens copied in, decode outputs copied back"}
+                      "note": "pinned host buffers: K, V and the newest query copied in first; Q copied in and O copied "
+                              "back in row ranges on two copy streams while tca_attn_prefill_rows computes the "
+                              "ranges already present; decode tokens copied in, decode outputs copied back; the "
+                              "timed prefill ends when the last range of O has reached the host",
+                      "row_ranges": len(pipe.row_ranges)}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = time_oracle(wl_rank, data, p)

@@ -191,6 +191,22 @@ int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const 
                      void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same attention (Eq. 2) for the query rows [row_begin, row_end) of every head only; the
+ * other rows of O are not touched.  A row's result does not depend on which call computed it:
+ * calls over a partition of [0, L) leave O bit-identical to one tca_attn_prefill call.  It
+ * lets a caller whose Q arrives (or whose O leaves) in pieces overlap the transfers with the
+ * arithmetic.  Q, K, V, O, L, cache and ws are those of tca_attn_prefill (Q and O are still
+ * addressed as the full [batch, n_q_heads, L, d] arrays); row_begin must be a multiple of
+ * TCA_PREFILL_ROW_ALIGN, 0 <= row_begin < row_end <= L, else TCA_ERR_INVALID_ARG.  Calls that
+ * may run concurrently need a workspace each.
+ */
+#define TCA_PREFILL_ROW_ALIGN 128
+int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, const void* V,
+                          int64_t L, int64_t row_begin, int64_t row_end,
+                          const tca_cache_desc* cache, void* O,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/*
  * One decode step, Eq. 2 with a single query per head over the whole retained cache
  * (global region + tail ring) of its KV head.
  *   q  DEVICE [batch, n_q_heads, head_dim]     O  DEVICE out, same shape

@@ -29,7 +29,7 @@ TCA_STATE_WORDS = 8
 EXPORTS = (
     "tca_strerror", "tca_version", "tca_budget_resolve", "tca_workspace_bytes", "tca_score",
     "tca_select", "tca_cache_init", "tca_compact_kv", "tca_attn_prefill", "tca_attn_decode",
-    "tca_cache_append", "tca_ws_status", "tca_attn_decode_static",
+    "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
 )
 
 
@@ -80,6 +80,7 @@ def lib() -> C.CDLL:
         L.tca_cache_init.argtypes = [P, D, vp]
         L.tca_compact_kv.argtypes = [P, vp, vp, i64, vp, vp, vp, D, vp]
         L.tca_attn_prefill.argtypes = [P, vp, vp, vp, i64, D, vp, vp, sz, vp]
+        L.tca_attn_prefill_rows.argtypes = [P, vp, vp, vp, i64, i64, i64, D, vp, vp, sz, vp]
         L.tca_attn_decode.argtypes = [P, vp, D, vp, vp, sz, vp]
         L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
         L.tca_ws_status.argtypes = [vp, vp]
@@ -188,6 +189,12 @@ def tca_compact_kv(prm, K, V, L, idx, offsets_dev, offsets_host, cache: "Cache",
 def tca_attn_prefill(prm, Q, K, V, L, cache: "Cache", O, ws, stream=None) -> None:
     _check(lib().tca_attn_prefill(C.byref(prm), _dev(Q), _dev(K), _dev(V), L, C.byref(cache.desc), _dev(O),
                                   *_ws_args(ws), _stream(stream)), "tca_attn_prefill")
+
+
+def tca_attn_prefill_rows(prm, Q, K, V, L, row_begin, row_end, cache: "Cache", O, ws, stream=None) -> None:
+    _check(lib().tca_attn_prefill_rows(C.byref(prm), _dev(Q), _dev(K), _dev(V), L, row_begin, row_end,
+                                       C.byref(cache.desc), _dev(O), *_ws_args(ws), _stream(stream)),
+           "tca_attn_prefill_rows")
 
 
 def tca_attn_decode(prm, q, cache: "Cache", O, ws, stream=None) -> None:

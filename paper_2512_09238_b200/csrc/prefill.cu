@@ -1,26 +1,28 @@
-// tca_attn_prefill: entry point of the sparse causal prefill attention (Eq. 2).
+// tca_attn_prefill / tca_attn_prefill_rows: entry points of the sparse causal prefill attention (Eq. 2).
 // fp32 inputs run on the FP32 pipes; bf16 inputs run on the tcgen05 tensor-core kernel
 // unless TCA_FLAG_PREFILL_SIMT asks for the FP32-pipe reference kernel.
 #include "common.cuh"
 
 namespace tca {
 template <typename T, int D>
-int launch_prefill_simt(const tca_params*, const void*, const void*, const void*, int64_t,
+int launch_prefill_simt(const tca_params*, const void*, const void*, const void*, int64_t, int64_t, int64_t,
                         const tca_cache_desc*, void*, cudaStream_t);
 template <int D>
-int launch_prefill_tc(const tca_params*, const void*, const void*, const void*, int64_t, const tca_cache_desc*,
-                      void*, void*, cudaStream_t);
+int launch_prefill_tc(const tca_params*, const void*, const void*, const void*, int64_t, int64_t, int64_t,
+                      const tca_cache_desc*, void*, void*, cudaStream_t);
 }  // namespace tca
 
 using namespace tca;
 
-extern "C" int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
-                                const tca_cache_desc* c, void* O, void* ws, size_t ws_bytes, void* stream) {
+extern "C" int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
+                                     int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O,
+                                     void* ws, size_t ws_bytes, void* stream) {
   int st = check_params(prm);
   if (st != TCA_OK) return st;
   TCA_CHECK_ARG(Q && K && V && c && O && ws);
   TCA_CHECK_ARG(c->k && c->v && c->pos && c->state);
   TCA_CHECK_ARG(L >= 1 && L < (int64_t(1) << 31));
+  TCA_CHECK_ARG(row_begin >= 0 && row_begin < row_end && row_end <= L && row_begin % TCA_PREFILL_ROW_ALIGN == 0);
   TCA_CHECK_ARG(prm->window >= 1);  // a query always sees itself through its local subset
   TCA_CHECK_ARG(aligned(Q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(O, 16) && aligned(ws, 256));
   TCA_CHECK_ARG(aligned(c->k, 16) && aligned(c->v, 16));
@@ -31,14 +33,19 @@ extern "C" int tca_attn_prefill(const tca_params* prm, const void* Q, const void
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return TCA_ERR_CUDA;  // status word
   if (prm->dtype == TCA_F32) {
-    if (prm->head_dim == 128) return launch_prefill_simt<float, 128>(prm, Q, K, V, L, c, O, s);
-    return launch_prefill_simt<float, 64>(prm, Q, K, V, L, c, O, s);
+    if (prm->head_dim == 128) return launch_prefill_simt<float, 128>(prm, Q, K, V, L, row_begin, row_end, c, O, s);
+    return launch_prefill_simt<float, 64>(prm, Q, K, V, L, row_begin, row_end, c, O, s);
   }
   if (prm->flags & TCA_FLAG_PREFILL_SIMT) {
-    if (prm->head_dim == 128) return launch_prefill_simt<__nv_bfloat16, 128>(prm, Q, K, V, L, c, O, s);
-    return launch_prefill_simt<__nv_bfloat16, 64>(prm, Q, K, V, L, c, O, s);
+    if (prm->head_dim == 128) return launch_prefill_simt<__nv_bfloat16, 128>(prm, Q, K, V, L, row_begin, row_end, c, O, s);
+    return launch_prefill_simt<__nv_bfloat16, 64>(prm, Q, K, V, L, row_begin, row_end, c, O, s);
   }
   TCA_CHECK_ARG(c->seg_start && c->n_global);
-  if (prm->head_dim == 128) return launch_prefill_tc<128>(prm, Q, K, V, L, c, O, ws, s);
-  return launch_prefill_tc<64>(prm, Q, K, V, L, c, O, ws, s);
+  if (prm->head_dim == 128) return launch_prefill_tc<128>(prm, Q, K, V, L, row_begin, row_end, c, O, ws, s);
+  return launch_prefill_tc<64>(prm, Q, K, V, L, row_begin, row_end, c, O, ws, s);
+}
+
+extern "C" int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
+                                const tca_cache_desc* c, void* O, void* ws, size_t ws_bytes, void* stream) {
+  return tca_attn_prefill_rows(prm, Q, K, V, L, 0, L, c, O, ws, ws_bytes, stream);
 }

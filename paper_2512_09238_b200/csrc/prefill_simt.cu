@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kPfThreads)
 prefill_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* __restrict__ V, int64_t L,
                     const T* __restrict__ Kc, const T* __restrict__ Vc, const int32_t* __restrict__ pos,
                     const int64_t* __restrict__ state, int n_q_heads, int n_kv_heads, int window, int64_t mb,
-                    float scale_log2e, T* __restrict__ O) {
+                    float scale_log2e, T* __restrict__ O, int tile0) {
   constexpr int LD = PfSmem<D>::LD, LDP = PfSmem<D>::LDP;
   constexpr int NC = D / 64;  // 4-wide output column chunks per thread
   extern __shared__ __align__(16) float smem[];
@@ -78,7 +78,7 @@ prefill_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int hq = blockIdx.y;
   const int n_tiles = gridDim.x;
-  const int tile = n_tiles - 1 - blockIdx.x;  // longest rows first
+  const int tile = tile0 + n_tiles - 1 - blockIdx.x;  // longest rows first
   const int seq = hq / n_q_heads;
   const int G = n_q_heads / n_kv_heads;
   const int u = seq * n_kv_heads + (hq % n_q_heads) / G;
@@ -241,27 +241,30 @@ prefill_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
 
 template <typename T, int D>
 int launch_prefill_simt(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
-                        const tca_cache_desc* c, void* O, cudaStream_t stream) {
+                        int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O, cudaStream_t stream) {
   auto kern = prefill_simt_kernel<T, D>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(PfSmem<D>::bytes)) !=
       cudaSuccess)
     return TCA_ERR_CUDA;
   const int64_t mb = num_blocks(prm, L) * prm->block;
-  dim3 grid(unsigned((L + kPfBM - 1) / kPfBM), unsigned(prm->batch * prm->n_q_heads));
+  const int tile0 = int(row_begin / kPfBM);
+  dim3 grid(unsigned((row_end - row_begin + kPfBM - 1) / kPfBM), unsigned(prm->batch * prm->n_q_heads));
   kern<<<grid, kPfThreads, PfSmem<D>::bytes, stream>>>(
       static_cast<const T*>(Q), static_cast<const T*>(K), static_cast<const T*>(V), L,
       static_cast<const T*>(c->k), static_cast<const T*>(c->v), c->pos, c->state, prm->n_q_heads,
-      prm->n_kv_heads, prm->window, mb, prm->sm_scale * 1.4426950408889634f, static_cast<T*>(O));
+      prm->n_kv_heads, prm->window, mb, prm->sm_scale * 1.4426950408889634f, static_cast<T*>(O), tile0);
   return check_launch();
 }
 
 template int launch_prefill_simt<float, 64>(const tca_params*, const void*, const void*, const void*, int64_t,
-                                            const tca_cache_desc*, void*, cudaStream_t);
+                                            int64_t, int64_t, const tca_cache_desc*, void*, cudaStream_t);
 template int launch_prefill_simt<float, 128>(const tca_params*, const void*, const void*, const void*, int64_t,
-                                             const tca_cache_desc*, void*, cudaStream_t);
+                                             int64_t, int64_t, const tca_cache_desc*, void*, cudaStream_t);
 template int launch_prefill_simt<__nv_bfloat16, 64>(const tca_params*, const void*, const void*, const void*,
-                                                    int64_t, const tca_cache_desc*, void*, cudaStream_t);
+                                                    int64_t, int64_t, int64_t, const tca_cache_desc*, void*,
+                                                    cudaStream_t);
 template int launch_prefill_simt<__nv_bfloat16, 128>(const tca_params*, const void*, const void*, const void*,
-                                                     int64_t, const tca_cache_desc*, void*, cudaStream_t);
+                                                     int64_t, int64_t, int64_t, const tca_cache_desc*, void*,
+                                                     cudaStream_t);
 
 }  // namespace tca

@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restrict__ pos,
                   const int64_t* __restrict__ state, int64_t L, int n_q_heads, int n_kv_heads, int window,
                   int64_t mb, float scale_log2e, __nv_bfloat16* __restrict__ O, int* __restrict__ status,
-                  int n_qtiles, int pairs_per_unit) {
+                  int n_qtiles, int pairs_per_unit, int tile0) {
   using Cfg = TcCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -101,7 +101,7 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
   const int per_unit = n_qtiles * pairs_per_unit;
   const int u = int(blockIdx.x) / per_unit;
   const int rem = int(blockIdx.x) % per_unit;
-  const int tile = n_qtiles - 1 - rem / pairs_per_unit;
+  const int tile = tile0 + n_qtiles - 1 - rem / pairs_per_unit;
   const int pair = rem % pairs_per_unit;
   const int nh = min(2, G - 2 * pair);                          // heads handled here
   const int seq = u / n_kv_heads, kvh = u % n_kv_heads;
@@ -409,7 +409,8 @@ size_t prefill_tc_ws_bytes(const tca_params* prm) {
 
 template <int D>
 int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
-                      const tca_cache_desc* c, void* O, void* ws, cudaStream_t stream) {
+                      int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O, void* ws,
+                      cudaStream_t stream) {
   using Cfg = TcCfg<D>;
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int G = prm->n_q_heads / prm->n_kv_heads;
@@ -429,20 +430,21 @@ int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const
                                  stream));
   auto kern = prefill_tc_kernel<D>;
   TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::bytes));
-  const int n_qtiles = int((L + BM - 1) / BM);
+  const int tile0 = int(row_begin / BM);
+  const int n_qtiles = int((row_end - row_begin + BM - 1) / BM);
   const int pairs = (G + 1) / 2;
   const int64_t n_ctas = int64_t(n_qtiles) * U * pairs;
   if (n_ctas >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;
   const int64_t mb = num_blocks(prm, L) * prm->block;
   kern<<<unsigned(n_ctas), kThreads, Cfg::bytes, stream>>>(
       maps_dev, c->pos, c->state, L, prm->n_q_heads, prm->n_kv_heads, prm->window, mb,
-      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs);
+      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs, tile0);
   return check_launch();
 }
 
-template int launch_prefill_tc<64>(const tca_params*, const void*, const void*, const void*, int64_t,
-                                   const tca_cache_desc*, void*, void*, cudaStream_t);
-template int launch_prefill_tc<128>(const tca_params*, const void*, const void*, const void*, int64_t,
-                                    const tca_cache_desc*, void*, void*, cudaStream_t);
+template int launch_prefill_tc<64>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
+                                   int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
+template int launch_prefill_tc<128>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
+                                    int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
 
 }  // namespace tca

@@ -127,6 +127,33 @@ def test_prefill_matches_oracle_on_every_row(runs, name):
                 H.check_attention(out[s, h * G + g], want, wl.dtype, f"{name} seq {s} head {h * G + g}")
 
 
+@pytest.mark.parametrize("name", ["config1", "bf16_gqa4", "bf16_g7"])
+def test_prefill_by_row_ranges_is_bit_identical(runs, name):
+    """Row ranges that partition [0, L), in any order, each with its own workspace, leave O equal
+    bit for bit to the single call; rows outside a range are not written."""
+    wl, data, p, run, oracle = runs(name)
+    whole = H.gpu_prefill(run)
+    L = run.L
+    cuts = sorted({0, 128, 384, min(L, 1280), L})
+    cuts = [c for c in cuts if c <= L]
+    parts = list(zip(cuts[:-1], cuts[1:]))
+    out = torch.full_like(run.dev["q"], float("nan"))
+    first = parts[-1]                                         # the last range first: order must not matter
+    for (r0, r1) in [first] + parts[:-1]:
+        ws = B.alloc_workspace(run.prm, L, B.TCA_OP_PREFILL)
+        B.tca_attn_prefill_rows(run.prm, run.dev["q"], run.dev["k"], run.dev["v"], L, r0, r1, run.cache, out, ws)
+        assert B.tca_ws_status(ws) == B.TCA_OK
+        if (r0, r1) == first and len(parts) > 1:              # nothing below r0 has been written yet
+            assert torch.isnan(out[:, :, :r0].float()).all()
+    a, b = whole.view(torch.uint8), out.view(torch.uint8)
+    assert torch.equal(a, b)
+    ws = B.alloc_workspace(run.prm, L, B.TCA_OP_PREFILL)
+    for bad in [(64, 128), (0, L + 1), (128, 128), (-128, 128)]:
+        with pytest.raises(B.TcaError):
+            B.tca_attn_prefill_rows(run.prm, run.dev["q"], run.dev["k"], run.dev["v"], L, bad[0], bad[1], run.cache,
+                                    out, ws)
+
+
 @pytest.mark.parametrize("name", ["bf16_gqa4", "bf16_d64_g2", "bf16_g7"])
 def test_bf16_prefill_reference_kernel_agrees(runs, name):
     """The FP32-pipe kernel and the default bf16 kernel see the same inputs."""
