@@ -27,7 +27,9 @@ notes with its justification):
   * the run lengths of Psi are floor(m * p_k) plus a largest-remainder correction so
     that Psi has exactly m entries;
   * ties inside Top(t; B) go to the lower token index;
-  * decoding: the block that leaves the window is the one compressed.
+  * decoding: the block that leaves the window is the one compressed;
+  * Algorithm 1: column means over the causally visible rows; the aggregated score is taken
+    as a share of its value at a 100 % budget; no valid candidate => the last candidate.
 
 Parity pins (tests/test_oracle_pins.py): dense causal attention by an independent
 brute force at 100 % budget and at w >= L; masked attention against an independently
@@ -51,7 +53,7 @@ __all__ = [
     "budget_map", "mean_retain_floor", "rank_blocks", "block_requirement",
     "select_tokens", "retained_set", "select_head", "visible_mask_row",
     "attention_rows", "attention_over_set", "candidate_grid", "DecodeCache",
-    "dropped_mass",
+    "dropped_mass", "attention_column_means", "aggregated_score", "calibrate_head",
 ]
 
 
@@ -253,6 +255,74 @@ def candidate_grid(b: int, M: int = 14, sigma: float = 1.0) -> np.ndarray:
         phi = np.exp(-((x - mu) ** 2) / (2.0 * sigma * sigma))
         rows.append(phi / phi.sum())
     return np.stack(rows)
+
+
+# ----------------------------------------------------------------------------- Algorithm 1 (offline)
+def attention_column_means(Q: np.ndarray, K: np.ndarray, sm_scale: float) -> np.ndarray:
+    """Inner term of Eq. 4: c[k] = mean over the non-zero entries of column k of A.
+
+    A = softmax(Q K^T sm_scale) with the causal mask (reading R1), so the non-zero entries of
+    column k are the rows j >= k and there are L - k of them.  Q is [G, L, d] (the query heads
+    that share the KV head; G = 1 for plain multi-head attention); the result is the mean of
+    the G heads' columns, the same aggregation as for the importance of Eq. 5.  Returns [L].
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    if Q.ndim == 2:
+        Q = Q[None]
+    G, L, _ = Q.shape
+    col = np.zeros(L, dtype=np.float64)
+    for g in range(G):
+        for j in range(L):
+            x = (K[:j + 1] @ Q[g, j]) * sm_scale
+            x -= x.max()
+            e = np.exp(x)
+            col[:j + 1] += e / e.sum()
+    return col / (G * (L - np.arange(L, dtype=np.float64)))
+
+
+def aggregated_score(S: np.ndarray, c: np.ndarray, n_candidates: int) -> float:
+    """a_i of Eq. 4 for the selected set S, as a share of what selecting every candidate gives.
+
+    Eq. 4 is the plain sum of c over S.  The threshold tau of Algorithm 1 is "a share of the
+    aggregated attention mass", and the plain sum is not bounded by 1 (it depends on L and on how
+    local the head is), so the sum is divided by its value for S = all candidates [0, m*b): the
+    100 % configuration then scores exactly 1.
+    """
+    total = float(np.sum(c[:n_candidates]))
+    return float(np.sum(c[np.asarray(S, dtype=np.int64)])) / total if total > 0.0 else 1.0
+
+
+def calibrate_head(Q: np.ndarray, K: np.ndarray, candidates: np.ndarray, b: int, w: int, alpha: float,
+                   tau: float, sm_scale: float):
+    """Algorithm 1 for one KV head: the sparsest candidate that keeps a share tau of the score.
+
+    For every candidate p^i the online selection (Eq. 5-8 with the newest query, exactly as at
+    inference) gives S_i; a_i follows Eq. 4; among the candidates with a_i >= tau the one with the
+    fewest selected tokens wins (the lowest index on a tie).  If no candidate reaches tau the last
+    one (the most accurate end of the sweep) is returned.  Returns (choice, a [M], sizes [M]).
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    if Q.ndim == 2:
+        Q = Q[None]
+    L = K.shape[0]
+    m = num_blocks(L, b, w)
+    c = attention_column_means(Q, K, sm_scale)
+    log_s = log_importance(Q[:, L - 1], K, sm_scale)
+    h = block_metric(log_s, m, b, alpha)
+    M = len(candidates)
+    a = np.zeros(M, dtype=np.float64)
+    sizes = np.zeros(M, dtype=np.int64)
+    for i in range(M):
+        t = block_requirement(h, resolve_counts(candidates[i], m), b)
+        S = select_tokens(log_s, t, b)
+        a[i] = aggregated_score(S, c, m * b)
+        sizes[i] = len(S)
+    valid = np.nonzero(a >= tau)[0]
+    if len(valid) == 0:
+        return M - 1, a, sizes
+    choice = int(valid[np.argmin(sizes[valid])])      # argmin returns the first minimum: lowest index
+    return choice, a, sizes
 
 
 # ----------------------------------------------------------------------------- steps 8-9: decoding

@@ -367,3 +367,72 @@ def test_candidate_grid_closed_forms(golden):
     # budgets grow monotonically from efficiency- to accuracy-oriented
     mean_keep = C @ O.retain_counts(b)
     assert np.all(np.diff(mean_keep) > 0)
+
+
+# ----------------------------------------------------------------------------- Algorithm 1 / Eq. 4
+def test_column_means_closed_form_for_uniform_attention():
+    """q = 0 makes every causal row uniform, A[j, k] = 1/(j+1), so the mean of column k over its
+    L - k non-zero rows is (H_L - H_k)/(L - k) with H the harmonic numbers."""
+    L, d = 37, 5
+    K = _rng(21).standard_normal((L, d))
+    c = O.attention_column_means(np.zeros((2, L, d)), K, 0.3)
+    H = np.concatenate([[0.0], np.cumsum(1.0 / np.arange(1, L + 1))])
+    np.testing.assert_allclose(c, (H[L] - H[:L]) / (L - np.arange(L)), rtol=1e-13)
+
+
+def test_column_means_against_a_masked_dense_matrix():
+    """Independent formulation: the full L x L matrix with a -inf upper triangle, SciPy's softmax
+    over rows, a column sum divided by the count of non-zero entries of that column."""
+    rng = _rng(22)
+    L, d, G = 29, 7, 3
+    Q, K = rng.standard_normal((G, L, d)) * 1.5, rng.standard_normal((L, d)) * 1.5
+    want = np.zeros(L)
+    for g in range(G):
+        X = (Q[g] @ K.T) * 0.4
+        X[np.triu_indices(L, 1)] = -np.inf
+        A = np.stack([sp_softmax(X[j]) for j in range(L)])
+        nnz = (A > 0).sum(0)
+        assert list(nnz) == list(L - np.arange(L))         # exactly the causally visible rows
+        want += A.sum(0) / nnz
+    np.testing.assert_allclose(O.attention_column_means(Q, K, 0.4), want / G, rtol=1e-12)
+    # every row of A sums to 1: weighting the means back by their counts gives L
+    c1 = O.attention_column_means(Q[:1], K, 0.4)
+    assert float(np.sum(c1 * (L - np.arange(L)))) == pytest.approx(L, rel=1e-12)
+
+
+def test_aggregated_score_is_a_share_of_the_full_selection():
+    c = np.array([0.5, 0.25, 0.125, 0.125, 9.0, 9.0])      # 4 candidates, 2 always-kept tail tokens
+    assert O.aggregated_score(np.arange(4), c, 4) == pytest.approx(1.0, rel=1e-15)
+    assert O.aggregated_score(np.array([0, 2]), c, 4) == pytest.approx(0.625, rel=1e-15)
+    assert O.aggregated_score(np.array([], dtype=np.int64), c, 4) == 0.0
+
+
+def test_calibration_picks_the_sparsest_candidate_that_reaches_tau():
+    """Two blocks of four tokens with a hand-made key layout: the newest query (and every other
+    query) looks almost only at token 1 of block 0 and token 2 of block 1.  Candidates: one token
+    per block, two per block, everything.  One token per block already holds more than 90 % of
+    the aggregated score, so Algorithm 1 must return it; with tau = 0.9999 only 'everything'
+    qualifies; sizes are 2, 4 and 8."""
+    b, w, d = 4, 4, 4
+    L = 2 * b + w
+    K = np.zeros((L, d))
+    K[1, 0] = K[6, 0] = 6.0                                 # the two keys every query likes
+    K[:, 1] = np.linspace(0.0, 0.3, L)                      # breaks ties inside the blocks
+    Q = np.zeros((1, L, d))
+    Q[0, :, 0] = 3.0
+    Q[0, :, 1] = 1.0
+    cands = np.array([[1.0, 0.0, 0.0], [0.0, 1.0, 0.0], [0.0, 0.0, 1.0]])   # over K = {1, 2, 4}
+    choice, a, sizes = O.calibrate_head(Q, K, cands, b, w, 0.5, 0.9, 1.0)
+    assert list(sizes) == [2, 4, 8]
+    assert a[2] == pytest.approx(1.0, rel=1e-12) and np.all(np.diff(a) > 0)
+    assert a[0] > 0.9 and choice == 0
+    # what candidate 0 selects is those two tokens, and a_0 is their share of the column means
+    r = O.select_head(Q[:, L - 1], K, cands[0], b, w, 0.5, 1.0)
+    assert list(r["S"]) == [1, 6]
+    c = O.attention_column_means(Q, K, 1.0)
+    assert a[0] == pytest.approx((c[1] + c[6]) / c[:8].sum(), rel=1e-12)
+    choice_hi, _, _ = O.calibrate_head(Q, K, cands, b, w, 0.5, 0.9999, 1.0)
+    assert choice_hi == 2
+    # a threshold nothing reaches falls back to the last candidate; equal sizes go to the lower index
+    assert O.calibrate_head(Q, K, cands[:2], b, w, 0.5, 0.99999, 1.0)[0] == 1
+    assert O.calibrate_head(Q, K, np.stack([cands[1], cands[1]]), b, w, 0.5, 0.5, 1.0)[0] == 0
