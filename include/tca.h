@@ -49,7 +49,7 @@ enum { TCA_FLAG_PREFILL_SIMT = 1 };
 
 enum {
   TCA_OP_SCORE = 0, TCA_OP_SELECT = 1, TCA_OP_COMPACT = 2,
-  TCA_OP_PREFILL = 3, TCA_OP_DECODE = 4, TCA_OP_APPEND = 5
+  TCA_OP_PREFILL = 3, TCA_OP_DECODE = 4, TCA_OP_APPEND = 5, TCA_OP_CALIB = 6
 };
 
 /* Hyper-parameters of one attention layer (Algorithm 2, REQUIRE line). */
@@ -205,6 +205,35 @@ int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, c
                           int64_t L, int64_t row_begin, int64_t row_end,
                           const tca_cache_desc* cache, void* O,
                           void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Offline calibration, Algorithm 1 and Eq. 4 (Section 4.1, "Cumulative-Score Configuration
+ * Determination").  It produces the per-head configuration p* that the functions above take
+ * as an input.  Three calls:
+ *
+ *   tca_calib_colmean  c[u][k] = mean over the causally visible rows j >= k (the non-zero
+ *                      entries of column k) of A = softmax(Q K^T * sm_scale), averaged over
+ *                      the G query heads of the KV head (the aggregation of tca_score).
+ *                      Q DEVICE [batch, n_q_heads, L, d], K DEVICE [batch, n_kv_heads, L, d],
+ *                      bf16 only (TCA_ERR_UNSUPPORTED otherwise); colmean DEVICE [U][L] doubles;
+ *                      ws DEVICE, tca_workspace_bytes(prm, L, TCA_OP_CALIB), word 0 is a status
+ *                      word readable with tca_ws_status.  prm->block and prm->window are not
+ *                      used.  Cost: two dense causal passes over Q K^T.
+ *   tca_calib_score    a[u] of Eq. 4 for the selection (idx, offsets_dev) that tca_select wrote
+ *                      for one candidate, as a share of the sum over all candidates [0, m*b):
+ *                      a 100 % budget scores exactly 1.  a_out DEVICE [U] doubles.
+ *   tca_calib_choose   HOST: the index of the candidate with the fewest selected tokens among
+ *                      those with a[i] >= tau (the lowest index on a tie); if none reaches tau,
+ *                      n_candidates - 1.  a, sizes HOST arrays of n_candidates entries.
+ *
+ * The caller runs tca_score once, then for every candidate p^i: tca_budget_resolve,
+ * tca_select, tca_calib_score; then tca_calib_choose per KV head.
+ */
+int tca_calib_colmean(const tca_params* prm, const void* Q, const void* K, int64_t L,
+                      double* colmean, void* ws, size_t ws_bytes, void* stream);
+int tca_calib_score(const tca_params* prm, const double* colmean, int64_t L,
+                    const int32_t* idx, const int64_t* offsets_dev, double* a_out, void* stream);
+int tca_calib_choose(const double* a, const int64_t* sizes, int n_candidates, double tau);
 
 /*
  * One decode step, Eq. 2 with a single query per head over the whole retained cache

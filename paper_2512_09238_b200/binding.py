@@ -23,13 +23,14 @@ TCA_ERR_CUDA, TCA_ERR_TIMEOUT, TCA_ERR_CAPACITY, TCA_ERR_SCRATCH_LIMIT = -4, -5,
 TCA_DECODE_STATIC_SCRATCH_BYTES = 16 << 20
 TCA_F32, TCA_BF16 = 0, 1
 TCA_FLAG_PREFILL_SIMT = 1
-TCA_OP_SCORE, TCA_OP_SELECT, TCA_OP_COMPACT, TCA_OP_PREFILL, TCA_OP_DECODE, TCA_OP_APPEND = range(6)
+TCA_OP_SCORE, TCA_OP_SELECT, TCA_OP_COMPACT, TCA_OP_PREFILL, TCA_OP_DECODE, TCA_OP_APPEND, TCA_OP_CALIB = range(7)
 TCA_STATE_WORDS = 8
 
 EXPORTS = (
     "tca_strerror", "tca_version", "tca_budget_resolve", "tca_workspace_bytes", "tca_score",
     "tca_select", "tca_cache_init", "tca_compact_kv", "tca_attn_prefill", "tca_attn_decode",
     "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
+    "tca_calib_colmean", "tca_calib_score", "tca_calib_choose",
 )
 
 
@@ -81,6 +82,9 @@ def lib() -> C.CDLL:
         L.tca_compact_kv.argtypes = [P, vp, vp, i64, vp, vp, vp, D, vp]
         L.tca_attn_prefill.argtypes = [P, vp, vp, vp, i64, D, vp, vp, sz, vp]
         L.tca_attn_prefill_rows.argtypes = [P, vp, vp, vp, i64, i64, i64, D, vp, vp, sz, vp]
+        L.tca_calib_colmean.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
+        L.tca_calib_score.argtypes = [P, vp, i64, vp, vp, vp, vp]
+        L.tca_calib_choose.argtypes = [vp, vp, C.c_int, C.c_double]
         L.tca_attn_decode.argtypes = [P, vp, D, vp, vp, sz, vp]
         L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
         L.tca_ws_status.argtypes = [vp, vp]
@@ -263,3 +267,22 @@ class Cache:
         ring = self.seg_start[u] + self.global_cap[u]
         t = ring + (self.tail_head[u] + np.arange(self.n_tail[u])) % self.tail_cap
         return np.concatenate([g, t]).astype(np.int64)
+
+
+def tca_calib_colmean(prm, Q, K, L, colmean, ws, stream=None) -> None:
+    _check(lib().tca_calib_colmean(C.byref(prm), _dev(Q), _dev(K), L, _dev(colmean), *_ws_args(ws), _stream(stream)),
+           "tca_calib_colmean")
+
+
+def tca_calib_score(prm, colmean, L, idx, offsets_dev, a_out, stream=None) -> None:
+    _check(lib().tca_calib_score(C.byref(prm), _dev(colmean), L, _dev(idx), _dev(offsets_dev), _dev(a_out),
+                                 _stream(stream)), "tca_calib_score")
+
+
+def tca_calib_choose(a: np.ndarray, sizes: np.ndarray, tau: float) -> int:
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    sizes = np.ascontiguousarray(sizes, dtype=np.int64)
+    r = lib().tca_calib_choose(a.ctypes.data, sizes.ctypes.data, len(a), float(tau))
+    if r < 0:
+        raise TcaError(r, "tca_calib_choose")
+    return int(r)

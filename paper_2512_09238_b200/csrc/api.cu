@@ -9,6 +9,7 @@
 namespace tca {
 
 size_t prefill_tc_ws_bytes(const tca_params* prm);
+size_t calib_ws_bytes(const tca_params* prm, int64_t L);
 
 int check_params(const tca_params* prm) {
   TCA_CHECK_ARG(prm != nullptr);
@@ -137,6 +138,7 @@ size_t tca_workspace_bytes(const tca_params* prm, int64_t L, int op) {
     case TCA_OP_PREFILL: return align_up(prefill_tc_ws_bytes(prm), 256);
     case TCA_OP_DECODE: return decode_ws_layout(prm, L, U, nullptr).bytes;
     case TCA_OP_APPEND: return 256;
+    case TCA_OP_CALIB: return prm->dtype == TCA_BF16 ? calib_ws_bytes(prm, L) : 0;
     default: return 0;
   }
 }

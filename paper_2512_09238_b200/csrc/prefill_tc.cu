@@ -33,6 +33,7 @@
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "tensor_map.cuh"
 
 namespace tca {
 namespace {
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restrict__ pos,
                   const int64_t* __restrict__ state, int64_t L, int n_q_heads, int n_kv_heads, int window,
                   int64_t mb, float scale_log2e, __nv_bfloat16* __restrict__ O, int* __restrict__ status,
-                  int n_qtiles, int pairs_per_unit, int tile0) {
+                  int n_qtiles, int pairs_per_unit, int tile0, float* __restrict__ lse_out, int64_t lse_stride) {
   using Cfg = TcCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -334,9 +335,12 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         if (ok) {
           ptx::tc_fence_after();
           const float inv = 1.f / l;
+          // minus the log2 of the row's softmax denominator, in the units of the scaled scores: the
+          // calibration pass adds it to a scaled score to get the log2 of a probability
+          if (lse_out != nullptr && i <= i_last) lse_out[size_t(hq0 + h) * lse_stride + size_t(i)] = -(m_used + log2f(l));
           __nv_bfloat16* orow = O + (size_t(hq0 + h) * L + size_t(i)) * D;
 #pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
+          for (int c = 0; c < D / 32 && O != nullptr; ++c) {
             uint32_t v[32];
             ptx::tmem_ld32(lane_addr + Cfg::colO(h) + c * 32, v);
             ptx::tc_wait_ld();
@@ -369,37 +373,6 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
 }
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// rows x D bf16 matrix (row-major, rows may be a [rows, heads] pair), boxes of 128 rows x 64 columns
-bool encode_map(CUtensorMap* out, const void* base, int D, int64_t rows, int64_t heads, int64_t head_stride_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(rows > 0 ? rows : 1), cuuint64_t(heads)};
-  cuuint64_t strides[2] = {cuuint64_t(D) * 2, cuuint64_t(head_stride_rows) * D * 2};
-  cuuint32_t box[3] = {64, 128, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  const cuuint32_t rank = heads > 0 ? 3 : 2;
-  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 size_t prefill_tc_ws_bytes(const tca_params* prm) {
@@ -410,7 +383,7 @@ size_t prefill_tc_ws_bytes(const tca_params* prm) {
 template <int D>
 int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
                       int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O, void* ws,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, float* lse_out, int64_t lse_stride) {
   using Cfg = TcCfg<D>;
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int G = prm->n_q_heads / prm->n_kv_heads;
@@ -438,13 +411,14 @@ int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const
   const int64_t mb = num_blocks(prm, L) * prm->block;
   kern<<<unsigned(n_ctas), kThreads, Cfg::bytes, stream>>>(
       maps_dev, c->pos, c->state, L, prm->n_q_heads, prm->n_kv_heads, prm->window, mb,
-      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs, tile0);
+      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs, tile0, lse_out,
+      lse_stride);
   return check_launch();
 }
 
 template int launch_prefill_tc<64>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
-                                   int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
+                                   int64_t, const tca_cache_desc*, void*, void*, cudaStream_t, float*, int64_t);
 template int launch_prefill_tc<128>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
-                                    int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
+                                    int64_t, const tca_cache_desc*, void*, void*, cudaStream_t, float*, int64_t);
 
 }  // namespace tca
