@@ -301,6 +301,56 @@ class Pipeline:
         }
 
 
+# ----------------------------------------------------------------------------- offline calibration (Algorithm 1)
+def calibration_leg(pipe, torch, B, sm_max_mhz, n_candidates: int = 14, tau: float = 0.9, reps: int = 2):
+    """Algorithm 1 on the prompt of the workload: column means of the causal attention map (two
+    dense passes on the tensor cores), then the 14 candidates of Eq. 3 through select + Eq. 4.
+    Not part of the timed step: it runs once per model, offline.  Reported against the MUFU
+    roof: one ex2 per (query, key) pair of each dense pass, 16 per clock and SM."""
+    wl, prm, L, U = pipe.wl, pipe.prm, pipe.L, pipe.U
+    col = torch.empty(U, L, dtype=torch.float64, device="cuda")
+    ws = B.alloc_workspace(prm, L, B.TCA_OP_CALIB)
+    B.tca_calib_colmean(prm, pipe.Qp, pipe.Kp, L, col, ws)          # warm-up
+    torch.cuda.synchronize()
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    e0.record()
+    for _ in range(reps):
+        B.tca_calib_colmean(prm, pipe.Qp, pipe.Kp, L, col, ws)
+    e1.record()
+    cands = B.tca_calib_candidates(wl.block, n_candidates, 1.0)
+    B.tca_score(prm, pipe.q_last, pipe.Kp, L, pipe.logscore, pipe.ws_score)
+    a_dev = torch.empty(n_candidates, U, dtype=torch.float64, device="cuda")
+    sizes = np.zeros((n_candidates, U), dtype=np.int64)
+    idx = torch.empty(max(1, U * pipe.m * wl.block), dtype=torch.int32, device="cuda")
+    for i in range(n_candidates):
+        n_k, n_sel, _ = B.tca_budget_resolve(np.tile(cands[i], (wl.n_kv_heads, 1)), pipe.m)
+        per_unit = np.tile(n_sel, wl.batch)
+        offsets = np.zeros(U + 1, dtype=np.int64)
+        offsets[1:] = np.cumsum(per_unit)
+        off_dev = torch.from_numpy(offsets).cuda()
+        B.tca_select(prm, pipe.logscore, L, n_k, idx, off_dev, None, None, pipe.ws_select)
+        B.tca_calib_score(prm, col, L, idx, off_dev, a_dev[i])
+        sizes[i] = per_unit
+    e2.record()
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(ws) == B.TCA_OK
+    a = a_dev.cpu().numpy()
+    choice = [B.tca_calib_choose(a[:, u], sizes[:, u], tau) for u in range(U)]
+    colmean_ms = e0.elapsed_time(e1) / reps
+    pairs = wl.batch * wl.n_q_heads * (L * (L + 1) // 2)            # causal (query, key) pairs, all heads
+    ex2_per_s = 2 * pairs / (colmean_ms * 1e-3)                     # both passes exponentiate every pair
+    peak = 16 * 148 * sm_max_mhz * 1e6
+    rows_sum = float((col[0] * (L - torch.arange(L, device="cuda", dtype=torch.float64))).sum().item())
+    return {"colmean_ms": colmean_ms, "candidates_ms": e1.elapsed_time(e2), "n_candidates": n_candidates, "tau": tau,
+            "choice_per_unit": choice,
+            "retained_share_of_candidates": [float(sizes[choice[u], u]) / (pipe.m * wl.block) for u in range(U)],
+            "a_of_choice": [float(a[choice[u], u]) for u in range(U)],
+            "row_sum_check_unit0": rows_sum / L,
+            "roofline": {"bound": "alu", "achieved": ex2_per_s / 1e12, "peak": peak / 1e12, "unit": "Tex2/s",
+                         "frac": ex2_per_s / peak,
+                         "peak_kind": "16 MUFU ex2 per clock and SM x 148 SMs x clocks.max.sm"}}
+
+
 # ----------------------------------------------------------------------------- oracle timing (CPU baseline)
 def time_oracle(wl, data, p, budget_s: float = 20.0):
     """The oracle as it stands on the host cores, on a bounded sample of the workload:
@@ -343,6 +393,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the 100 %-budget comparison run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-calibration", action="store_true", help="skip the offline calibration (Algorithm 1) leg")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -495,6 +546,9 @@ def main():
                               "ranges already present; decode tokens copied in, decode outputs copied back; the "
                               "timed prefill ends when the last range of O has reached the host",
                       "row_ranges": len(pipe.row_ranges)}
+
+    if rank == 0 and world == 1 and not args.no_calibration and wl.dtype == "bf16":
+        out["calibration"] = calibration_leg(pipe, torch, B, clocks.get("sm_max_mhz") or 1965.0)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = time_oracle(wl_rank, data, p)

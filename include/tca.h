@@ -236,6 +236,14 @@ int tca_calib_score(const tca_params* prm, const double* colmean, int64_t L,
 int tca_calib_choose(const double* a, const int64_t* sizes, int n_candidates, double tau);
 
 /*
+ * HOST: the candidate configurations of Eq. 3 (log-Gaussian over the retain counts 1, 2, 4, ...,
+ * block, centred at mu^i = log2(1 + (i-1)(block-1)/(M-1)), i = 1..M, fixed sigma).  p_out HOST
+ * [n_candidates][log2(block)+1] doubles, every row sums to 1.  block must be a power of two,
+ * n_candidates >= 2, sigma > 0, else TCA_ERR_INVALID_ARG.
+ */
+int tca_calib_candidates(int block, int n_candidates, double sigma, double* p_out);
+
+/*
  * One decode step, Eq. 2 with a single query per head over the whole retained cache
  * (global region + tail ring) of its KV head.
  *   q  DEVICE [batch, n_q_heads, head_dim]     O  DEVICE out, same shape

@@ -30,7 +30,7 @@ EXPORTS = (
     "tca_strerror", "tca_version", "tca_budget_resolve", "tca_workspace_bytes", "tca_score",
     "tca_select", "tca_cache_init", "tca_compact_kv", "tca_attn_prefill", "tca_attn_decode",
     "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
-    "tca_calib_colmean", "tca_calib_score", "tca_calib_choose",
+    "tca_calib_colmean", "tca_calib_score", "tca_calib_choose", "tca_calib_candidates",
 )
 
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.tca_calib_colmean.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
         L.tca_calib_score.argtypes = [P, vp, i64, vp, vp, vp, vp]
         L.tca_calib_choose.argtypes = [vp, vp, C.c_int, C.c_double]
+        L.tca_calib_candidates.argtypes = [C.c_int, C.c_int, C.c_double, vp]
         L.tca_attn_decode.argtypes = [P, vp, D, vp, vp, sz, vp]
         L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
         L.tca_ws_status.argtypes = [vp, vp]
@@ -286,3 +287,10 @@ def tca_calib_choose(a: np.ndarray, sizes: np.ndarray, tau: float) -> int:
     if r < 0:
         raise TcaError(r, "tca_calib_choose")
     return int(r)
+
+
+def tca_calib_candidates(block: int, n_candidates: int = 14, sigma: float = 1.0) -> np.ndarray:
+    nK = int(block).bit_length()
+    p = np.zeros((n_candidates, nK), dtype=np.float64)
+    _check(lib().tca_calib_candidates(block, n_candidates, float(sigma), p.ctypes.data), "tca_calib_candidates")
+    return p

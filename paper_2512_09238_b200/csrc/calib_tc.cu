@@ -23,6 +23,7 @@
 // workspace, lets outstanding copies land, frees TMEM and returns.
 #include <cuda.h>
 
+#include <cmath>
 #include <vector>
 
 #include "bulk_ring.cuh"
@@ -383,4 +384,23 @@ extern "C" int tca_calib_choose(const double* a, const int64_t* sizes, int n_can
   for (int i = 0; i < n_candidates; ++i)
     if (a[i] >= tau && (best < 0 || sizes[i] < sizes[best])) best = i;
   return best < 0 ? n_candidates - 1 : best;
+}
+
+extern "C" int tca_calib_candidates(int block, int n_candidates, double sigma, double* p_out) {
+  if (block < 1 || (block & (block - 1)) != 0 || n_candidates < 2 || !(sigma > 0.0) || !p_out)
+    return TCA_ERR_INVALID_ARG;
+  int nK = 1;
+  while ((1 << (nK - 1)) < block) ++nK;
+  for (int i = 0; i < n_candidates; ++i) {
+    // Eq. 3 with mu^i = log2(1 + (i - 1)(b - 1)/(M - 1)), i = 1..M
+    const double mu = std::log2(1.0 + double(i) * double(block - 1) / double(n_candidates - 1));
+    double sum = 0.0;
+    for (int k = 0; k < nK; ++k) {
+      const double x = double(k) - mu;               // log2 of the retain count 2^k, minus mu
+      p_out[size_t(i) * nK + k] = std::exp(-x * x / (2.0 * sigma * sigma));
+      sum += p_out[size_t(i) * nK + k];
+    }
+    for (int k = 0; k < nK; ++k) p_out[size_t(i) * nK + k] /= sum;
+  }
+  return TCA_OK;
 }

@@ -71,15 +71,15 @@ def test_column_means_match_the_oracle(name):
     assert torch.equal(col.view(torch.int64), again.view(torch.int64))
 
 
+@pytest.mark.parametrize("tau", [0.9, 0.5, 0.2])
 @pytest.mark.parametrize("name", ["gqa4_d128", "g2_d64"])
-def test_candidate_scores_and_choice_match_the_oracle(name):
+def test_candidate_scores_and_choice_match_the_oracle(name, tau):
     wl = CASES[name]
     data = I.generate(wl)
     prm, dev, col = _gpu_colmean(wl, data)
     L, U, G = wl.L, wl.batch * wl.n_kv_heads, wl.group
     m = (L - wl.window) // wl.block
     cands = O.candidate_grid(wl.block, 14, 1.0)
-    tau = 0.9
     logscore = torch.empty(U, L, dtype=torch.float64, device="cuda")
     q_last = dev["q"][:, :, L - 1, :].contiguous()
     B.tca_score(prm, q_last, dev["k"], L, logscore, B.alloc_workspace(prm, L, B.TCA_OP_SCORE))

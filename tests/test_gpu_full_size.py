@@ -196,3 +196,57 @@ def test_config5_budget_sweep_64k(frac):
     last = wl.decode_steps - 1
     want = cache.attend(I.widen(data["q"][s, h * G + 2, L + last]), Kw, Vw)
     H.check_attention(H.from_device(pipe.Od[last, s, h * G + 2]), want, wl.dtype, f"config5 decode f={frac}")
+
+
+def test_calibration_column_means_at_32k():
+    """Algorithm 1's dense passes at L = 32768 (config 3), checked through what holds at any size:
+    every row of the attention map sums to 1, so the column means weighted back by their counts
+    (L - k) sum to L for every KV head; sampled columns near the end, where only a few rows are
+    visible, against the oracle's definition evaluated for just those rows; Eq. 4 of the
+    all-candidates selection is exactly 1 and grows with the budget."""
+    wl = I.WORKLOADS["config3"]
+    data, p, pipe = _pipeline(wl)
+    L, U, G = wl.L, pipe.U, wl.group
+    col = torch.empty(U, L, dtype=torch.float64, device="cuda")
+    ws = B.alloc_workspace(pipe.prm, L, B.TCA_OP_CALIB)
+    B.tca_calib_colmean(pipe.prm, pipe.Qp, pipe.Kp, L, col, ws)
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(ws) == B.TCA_OK
+    c = col.cpu().numpy()
+    assert np.all(np.isfinite(c)) and np.all(c >= 0)
+    np.testing.assert_allclose((c * (L - np.arange(L))).sum(1), float(L), rtol=1e-5)
+    scale = H.scale_of(wl)
+    n_last = 96                                              # the last 96 rows see columns >= L - 96 fully
+    for u in (0, U - 1):
+        s, h = divmod(u, wl.n_kv_heads)
+        K = I.widen(data["k"][s, h, :L])
+        want = np.zeros(n_last)
+        for g in range(G):
+            Q = I.widen(data["q"][s, h * G + g, L - n_last:L])
+            for r in range(n_last):
+                j = L - n_last + r
+                x = (K[:j + 1] @ Q[r]) * scale
+                a = np.exp(x - x.max())
+                a /= a.sum()
+                want[:r + 1] += a[L - n_last:j + 1]
+        want /= G * (n_last - np.arange(n_last))
+        np.testing.assert_allclose(c[u, L - n_last:], want, rtol=2e-3, atol=1e-12)
+    # Eq. 4 for two budgets through the library's own selection
+    B.tca_score(pipe.prm, pipe.q_last, pipe.Kp, L, pipe.logscore, pipe.ws_score)
+    a_prev = None
+    for frac in (0.25, 1.0):
+        wlf = wl.scaled(budget=("fixed", frac))
+        n_k, n_sel, _ = B.tca_budget_resolve(I.budget_table(wlf), pipe.m)
+        offsets = np.zeros(U + 1, dtype=np.int64)
+        offsets[1:] = np.cumsum(np.tile(n_sel, wl.batch))
+        idx = torch.empty(int(offsets[-1]), dtype=torch.int32, device="cuda")
+        off_dev = torch.from_numpy(offsets).cuda()
+        B.tca_select(pipe.prm, pipe.logscore, L, n_k, idx, off_dev, None, None, pipe.ws_select)
+        a = torch.empty(U, dtype=torch.float64, device="cuda")
+        B.tca_calib_score(pipe.prm, col, L, idx, off_dev, a)
+        a = a.cpu().numpy()
+        assert np.all(a > 0) and np.all(a <= 1.0 + 1e-12)
+        if frac == 1.0:
+            np.testing.assert_allclose(a, 1.0, rtol=1e-12)
+            assert np.all(a >= a_prev)
+        a_prev = a

@@ -94,3 +94,21 @@ def test_workspace_sizes_scale_as_documented():
     assert score < 1.01 * 8 * 4 * L * 8 + (1 << 20)
     sel = B.tca_workspace_bytes(prm, L, B.TCA_OP_SELECT)
     assert sel >= 8 * 992 * 12
+
+
+def test_candidate_grid_host_helper_matches_eq3():
+    """Eq. 3 on the host side of the library against the oracle's restatement and its closed forms."""
+    for b in (2, 8, 32, 128):
+        got = B.tca_calib_candidates(b, 14, 1.0)
+        np.testing.assert_allclose(got, O.candidate_grid(b, 14, 1.0), rtol=1e-13, atol=1e-16)
+        np.testing.assert_allclose(got.sum(1), 1.0, rtol=1e-14)
+    g = B.tca_calib_candidates(128, 14, 1.0)
+    assert g[0, 1] / g[0, 0] == pytest.approx(np.exp(-0.5), rel=1e-12)      # mu^1 = 0
+    assert g[-1, -2] / g[-1, -1] == pytest.approx(np.exp(-0.5), rel=1e-12)  # mu^M = log2 b
+    for bad in ((96, 14, 1.0), (128, 1, 1.0), (128, 14, 0.0)):
+        with pytest.raises(B.TcaError):
+            B.tca_calib_candidates(*bad)
+    a = np.array([0.2, 0.91, 0.95])
+    assert B.tca_calib_choose(a, np.array([5, 9, 9]), 0.9) == 1
+    assert B.tca_calib_choose(a, np.array([5, 9, 7]), 0.9) == 2
+    assert B.tca_calib_choose(a, np.array([5, 9, 7]), 0.99) == 2            # none valid: the last candidate
