@@ -36,9 +36,12 @@ brute force at 100 % budget and at w >= L; masked attention against an independe
 built boolean mask; closed forms of the concentration term; a hand-worked selection
 example; the exact identity ||s - s~||_1 = 2*gamma behind Theorem 1; decode == last
 prefill row; invariants of the selection.  "Parity unpinned" against the authors' own
-implementation: GQA aggregation, the window/partition reading, the leftover rounding
-and the decode block choice -- the paper fixes none of them; they are pinned only to
-the readings above.
+implementation: GQA aggregation, the window/partition reading, the leftover rounding,
+the decode block choice, and for Algorithm 1 the normalisation of the aggregated score and
+the no-valid-candidate fall-back -- the paper fixes none of them; they are pinned only to
+the readings above.  Algorithm 1's column means are pinned by the harmonic-number closed
+form for uniform attention and by an independently masked dense matrix, its choice rule by a
+hand-worked example.
 """
 from __future__ import annotations
 
