@@ -168,7 +168,9 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
       }
     } else if (warp == 1) {
       // ------------------------------------------------------------- MMA issuer
-      if (lane == 0) {
+      // The whole warp runs this loop; one elected lane issues (see umma_ss_elect).  Waits are
+      // made warp-uniform so that the warp stays converged for elect.sync.
+      {
         constexpr uint32_t idescS = ptx::idesc_bf16(BM, BN, false);
         constexpr uint32_t idescPV = ptx::idesc_bf16(BM, D, true);
         const uint32_t q_base = ptx::smem_u32(smem + Cfg::offQ);
@@ -178,6 +180,9 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         const uint64_t dq = ptx::smem_desc_sw128(q_base, 16, 1024);
         const uint64_t dk = ptx::smem_desc_sw128(kv_base, 16, 1024);           // K tile as K-major B
         const uint64_t dv = ptx::smem_desc_sw128(kv_base, kHalfBytes, 1024);   // V tile as MN-major B
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+          return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
+        };
         auto issue_S = [&](int h, int slot) {
           const uint64_t a0 = dq + uint64_t(uint32_t(h * Cfg::kQ) >> 4);
           const uint64_t b0 = dk + uint64_t(uint32_t(slot * Cfg::kKV) >> 4);
@@ -185,7 +190,7 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t off = (uint32_t(kk >> 2) * kHalfBytes + uint32_t(kk & 3) * 32u) >> 4;
-            ptx::umma_ss(d, a0 + off, b0 + off, idescS, kk > 0);
+            ptx::umma_ss_elect(d, a0 + off, b0 + off, idescS, kk > 0);
           }
         };
         // O += P V with P read from TMEM (it overwrote the first 64 columns of S as packed bf16):
@@ -199,40 +204,41 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
           constexpr int kPer = BN / 16 / kPChunks;
 #pragma unroll
           for (int c = 0; c < kPChunks; ++c) {
-            if (!ptx::mbar_wait(&bars[BAR_P + h * kPChunks + c], parity, abort_flag)) return false;
+            if (!wait(&bars[BAR_P + h * kPChunks + c], parity)) return false;
             ptx::tc_fence_after();
 #pragma unroll
             for (int k2 = 0; k2 < kPer; ++k2) {
               const int kk = c * kPer + k2;
-              ptx::umma_ts(d, a + uint32_t(kk * 8), b0 + uint32_t((kk * 2048) >> 4), idescPV, (acc || kk > 0) ? 1u : 0u);
+              ptx::umma_ts_elect(d, a + uint32_t(kk * 8), b0 + uint32_t((kk * 2048) >> 4), idescPV,
+                                 (acc || kk > 0) ? 1u : 0u);
             }
           }
           return true;
         };
-        bool ok = ptx::mbar_wait(&bars[BAR_Q], 0, abort_flag) && ptx::mbar_wait(&bars[BAR_FULL + 0], 0, abort_flag);
+        bool ok = wait(&bars[BAR_Q], 0) && wait(&bars[BAR_FULL + 0], 0);
         if (ok) {
           ptx::tc_fence_after();
-          for (int h = 0; h < nh; ++h) { issue_S(h, 0); ptx::umma_commit(&bars[BAR_S + h]); }
-          ptx::umma_commit(&bars[BAR_EMPTY + 0]);
+          for (int h = 0; h < nh; ++h) { issue_S(h, 0); ptx::umma_commit_elect(&bars[BAR_S + h]); }
+          ptx::umma_commit_elect(&bars[BAR_EMPTY + 0]);
         }
         for (int t = 0; t < nt && ok; ++t) {
           const int nV = 2 * t + 1, slotV = nV % kRing;
           const int nK = 2 * t + 2, slotK = nK % kRing;
-          ok = ptx::mbar_wait(&bars[BAR_FULL + slotV], uint32_t(nV / kRing) & 1u, abort_flag);
+          ok = wait(&bars[BAR_FULL + slotV], uint32_t(nV / kRing) & 1u);
           for (int h = 0; h < nh && ok; ++h) {
             ok = issue_PV(h, slotV, t > 0, uint32_t(t) & 1u);
             if (!ok) break;
-            ptx::umma_commit(&bars[BAR_PV + h]);
-            if (h == nh - 1) ptx::umma_commit(&bars[BAR_EMPTY + slotV]);
+            ptx::umma_commit_elect(&bars[BAR_PV + h]);
+            if (h == nh - 1) ptx::umma_commit_elect(&bars[BAR_EMPTY + slotV]);
             if (t + 1 < nt) {
               if (h == 0) {
-                ok = ptx::mbar_wait(&bars[BAR_FULL + slotK], uint32_t(nK / kRing) & 1u, abort_flag);
+                ok = wait(&bars[BAR_FULL + slotK], uint32_t(nK / kRing) & 1u);
                 if (!ok) break;
                 ptx::tc_fence_after();
               }
               issue_S(h, slotK);
-              ptx::umma_commit(&bars[BAR_S + h]);
-              if (h == nh - 1) ptx::umma_commit(&bars[BAR_EMPTY + slotK]);
+              ptx::umma_commit_elect(&bars[BAR_S + h]);
+              if (h == nh - 1) ptx::umma_commit_elect(&bars[BAR_EMPTY + slotK]);
             }
           }
         }
