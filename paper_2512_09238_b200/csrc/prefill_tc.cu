@@ -18,11 +18,11 @@
 // TMEM (512 columns): S0 | S1 | O0 | O1; the bf16 P of a tile overwrites the first half of its
 // S columns and feeds the PV product straight from TMEM.  Shared memory: Q0 Q1 | 5-slot K/V ring.
 // Per tile the issuer runs  PV0(t) S0(t+1) PV1(t) S1(t+1)  so that S of one head is being
-// computed while the other head's softmax is in flight.  O stays in TMEM and is rescaled
+// computed while the other head's softmax is in flight; the whole issuer warp executes the
+// loop and an elected lane's tcgen05 instructions take effect (see umma_ss_elect).  O stays in TMEM and is rescaled
 // lazily: only when a row maximum grew by more than 2^8 since the last rescale.  The softmax
 // arithmetic uses the packed fp32x2 forms (fma, add) and the three-input max, which halves its
-// issue slots: the issuer thread shares a warp scheduler with two softmax warps and every slot
-// they take delays the next tcgen05.mma.  CTAs are ordered unit-major so that the CTAs resident
+// issue slots.  CTAs are ordered unit-major so that the CTAs resident
 // at one time read the same one or two KV heads out of L2.
 //
 // Every mbarrier wait is bounded; a wait that gives up raises the status word of the
@@ -224,21 +224,20 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         for (int t = 0; t < nt && ok; ++t) {
           const int nV = 2 * t + 1, slotV = nV % kRing;
           const int nK = 2 * t + 2, slotK = nK % kRing;
-          ok = wait(&bars[BAR_FULL + slotV], uint32_t(nV / kRing) & 1u);
+          const bool more = t + 1 < nt;
+          // everything a head's block needs is waited for first, then PV_h(t) and S_h(t+1) go to
+          // the tensor pipe back to back and the commits follow: nothing sits between the two
+          // products on the chain S -> softmax -> PV -> S
+          ok = wait(&bars[BAR_FULL + slotV], uint32_t(nV / kRing) & 1u) &&
+               (!more || wait(&bars[BAR_FULL + slotK], uint32_t(nK / kRing) & 1u));
           for (int h = 0; h < nh && ok; ++h) {
             ok = issue_PV(h, slotV, t > 0, uint32_t(t) & 1u);
             if (!ok) break;
-            ptx::umma_commit_elect(&bars[BAR_PV + h]);
-            if (h == nh - 1) ptx::umma_commit_elect(&bars[BAR_EMPTY + slotV]);
-            if (t + 1 < nt) {
-              if (h == 0) {
-                ok = wait(&bars[BAR_FULL + slotK], uint32_t(nK / kRing) & 1u);
-                if (!ok) break;
-                ptx::tc_fence_after();
-              }
-              issue_S(h, slotK);
-              ptx::umma_commit_elect(&bars[BAR_S + h]);
-              if (h == nh - 1) ptx::umma_commit_elect(&bars[BAR_EMPTY + slotK]);
+            if (more) issue_S(h, slotK);
+            ptx::umma_commit_elect(&bars[more ? BAR_S + h : BAR_PV + h]);   // S ready implies PV done
+            if (h == nh - 1) {
+              ptx::umma_commit_elect(&bars[BAR_EMPTY + slotV]);
+              if (more) ptx::umma_commit_elect(&bars[BAR_EMPTY + slotK]);
             }
           }
         }
@@ -337,7 +336,7 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
           }
         }
         // epilogue: O / l -> bf16 -> global
-        if (ok) ok = ptx::mbar_wait(&bars[BAR_PV + h], uint32_t(nt - 1) & 1u, abort_flag);
+        if (ok) ok = ptx::mbar_wait(&bars[BAR_PV + h], 0, abort_flag);   // committed once, after the last PV
         if (ok) {
           ptx::tc_fence_after();
           const float inv = 1.f / l;
