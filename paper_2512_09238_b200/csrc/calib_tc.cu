@@ -136,12 +136,15 @@ calib_colsum_kernel(const CUtensorMap* __restrict__ maps, const float* __restric
         }
       }
     } else if (warp == 1) {
-      // ------------------------------------------------------------- MMA issuer
-      if (lane == 0) {
+      // ------------------------------------------------------------- MMA issuer (whole warp, elected lane)
+      {
         constexpr uint32_t idesc = ptx::idesc_bf16(CT, CT, false);
         const uint64_t dk = ptx::smem_desc_sw128(ptx::smem_u32(smem + Cfg::offK), 16, 1024);        // keys as A
         const uint64_t dq = ptx::smem_desc_sw128(ptx::smem_u32(smem + Cfg::offRing), 16, 1024);     // queries as B
-        bool ok = ptx::mbar_wait(&bars[CB_K], 0, abort_flag);
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+          return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
+        };
+        bool ok = wait(&bars[CB_K], 0);
         int jj = 0;
         uint32_t done[2] = {0u, 0u};                 // tiles issued so far per chain
         for (int n = 0; n < n_items && ok; ++n) {
@@ -149,8 +152,8 @@ calib_colsum_kernel(const CUtensorMap* __restrict__ maps, const float* __restric
           for (int c = 0; c < 2; ++c) {
             if (2 * pair + c >= G) continue;
             const int slot = jj % kQRing;
-            ok = ptx::mbar_wait(&bars[CB_FULL + slot], uint32_t(jj / kQRing) & 1u, abort_flag) &&
-                 (done[c] == 0 || ptx::mbar_wait(&bars[CB_FREE + c], (done[c] - 1) & 1u, abort_flag));
+            ok = wait(&bars[CB_FULL + slot], uint32_t(jj / kQRing) & 1u) &&
+                 (done[c] == 0 || wait(&bars[CB_FREE + c], (done[c] - 1) & 1u));
             if (!ok) break;
             ptx::tc_fence_after();
             const uint64_t b0 = dq + uint64_t(uint32_t(slot * Cfg::kSlot) >> 4);
@@ -158,10 +161,10 @@ calib_colsum_kernel(const CUtensorMap* __restrict__ maps, const float* __restric
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t off = (uint32_t(kk >> 2) * kColHalfBytes + uint32_t(kk & 3) * 32u) >> 4;
-              ptx::umma_ss(d, dk + off, b0 + off, idesc, kk > 0);
+              ptx::umma_ss_elect(d, dk + off, b0 + off, idesc, kk > 0);
             }
-            ptx::umma_commit(&bars[CB_S + c]);
-            ptx::umma_commit(&bars[CB_EMPTY + slot]);
+            ptx::umma_commit_elect(&bars[CB_S + c]);
+            ptx::umma_commit_elect(&bars[CB_EMPTY + slot]);
             ++done[c];
             ++jj;
           }
