@@ -42,7 +42,7 @@ def scale_of(wl: I.Workload) -> float:
 
 
 @dataclass
-class GpuRun:
+class DeviceRun:
     prm: B.tca_params
     wl: I.Workload
     L: int
@@ -60,7 +60,7 @@ class GpuRun:
 
 
 def gpu_select_compact(wl: I.Workload, data: Dict[str, np.ndarray], p: np.ndarray, L: Optional[int] = None,
-                       extra_blocks: int = 0, flags: int = 0) -> GpuRun:
+                       extra_blocks: int = 0, flags: int = 0) -> DeviceRun:
     """score -> select -> compact on the GPU for the first L tokens of `data`."""
     L = wl.L if L is None else L
     prm = params_for(wl, flags)
@@ -83,10 +83,10 @@ def gpu_select_compact(wl: I.Workload, data: Dict[str, np.ndarray], p: np.ndarra
     cache = B.Cache(prm, per_unit + extra_blocks * tk, wl.window + wl.block, tk)
     B.tca_compact_kv(prm, dev["k"], dev["v"], L, idx, offsets_dev, offsets, cache)
     torch.cuda.synchronize()
-    return GpuRun(prm, wl, L, m, n_k, n_sel, tbar, offsets, logscore, h, t, idx, cache, dev)
+    return DeviceRun(prm, wl, L, m, n_k, n_sel, tbar, offsets, logscore, h, t, idx, cache, dev)
 
 
-def gpu_prefill(run: GpuRun) -> torch.Tensor:
+def gpu_prefill(run: DeviceRun) -> torch.Tensor:
     O_dev = torch.empty_like(run.dev["q"])
     ws = B.alloc_workspace(run.prm, run.L, B.TCA_OP_PREFILL)
     B.tca_attn_prefill(run.prm, run.dev["q"], run.dev["k"], run.dev["v"], run.L, run.cache, O_dev, ws)
@@ -94,7 +94,7 @@ def gpu_prefill(run: GpuRun) -> torch.Tensor:
     return O_dev
 
 
-def gpu_decode(run: GpuRun, q: torch.Tensor) -> torch.Tensor:
+def gpu_decode(run: DeviceRun, q: torch.Tensor) -> torch.Tensor:
     out = torch.empty_like(q)
     ws = B.alloc_workspace(run.prm, run.cache.rows_total, B.TCA_OP_DECODE)
     B.tca_attn_decode(run.prm, q, run.cache, out, ws)
