@@ -406,11 +406,18 @@ def main():
         wl = wl.scaled(L=args.length)
     if args.decode_steps >= 0:
         wl = wl.scaled(decode_steps=args.decode_steps)
+    elt_bytes = 2 if wl.dtype == "bf16" else 4
+    qo_mib = wl.batch * wl.n_q_heads * wl.L * wl.head_dim * elt_bytes / 2 ** 20
+    if qo_mib > 126:
+        l2_note = (f"inputs larger than L2 (Q and O are {qo_mib:.0f} MiB each; a decode step streams the whole "
+                   "retained cache)")
+    else:
+        l2_note = f"inputs smaller than L2 (Q is {qo_mib:.1f} MiB): a parity-size workload, not a bench line"
     config = {"workload": f"{wl.name}: 1 attention layer, {wl.n_q_heads}/{wl.n_kv_heads} heads, d={wl.head_dim}, "
                           f"{wl.dtype}, batch {wl.batch}, causal prefill L={wl.L} with selection and compaction, "
                           f"then {wl.decode_steps} decode steps (append + attend)",
               "block": wl.block, "window": wl.window, "alpha": wl.alpha, "seed": wl.seed,
-              "l2": "inputs larger than L2 (Q and O are 1 GiB each; a decode step streams the whole retained cache)",
+              "l2": l2_note,
               "parallelism": "replicas only" if world > 1 else "1 GPU"}
 
     if args.impl == "reference":
