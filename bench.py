@@ -487,7 +487,7 @@ def main():
     work = pipe.algorithmic_work()
     prefill_ms = stages["score"] + stages["select"] + stages["compact"] + stages["prefill"]
     value = job_throughput(world, wl.batch, wl.L, prefill_ms)
-    decode_us = stages["decode"] * 1e3 / max(1, wl.decode_steps)
+    decode_us = stages["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None   # no decode phase: no figure
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -514,7 +514,7 @@ def main():
         "select": {"ms": stages["select"]},
         "compact": hbm_stage(work["compact_bytes"], stages["compact"]),
         "prefill": {"ms": stages["prefill"], "flops": work["prefill_flops"], "dense_flops": work["dense_prefill_flops"]},
-        "decode_step": hbm_stage(work["decode_bytes_per_step"], decode_us * 1e-3),
+        "decode_step": hbm_stage(work["decode_bytes_per_step"], decode_us * 1e-3) if decode_us else None,
         "retained_fraction": work["retained_fraction"],
         "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
     }
@@ -526,10 +526,10 @@ def main():
         pipe = Pipeline(dense_wl, data, I.budget_table(dense_wl), torch, B, host_io=False)
         _, st_dense, _ = timed(host_io=False)
         dense_prefill = st_dense["score"] + st_dense["select"] + st_dense["compact"] + st_dense["prefill"]
-        dense_decode_us = st_dense["decode"] * 1e3 / max(1, wl.decode_steps)
+        dense_decode_us = st_dense["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None
         out["dense_baseline"] = {"budget": 1.0, "prefill_ms": dense_prefill, "decode_us_per_step": dense_decode_us,
                                  "speedup_prefill": dense_prefill / prefill_ms,
-                                 "speedup_decode": dense_decode_us / decode_us if decode_us > 0 else None,
+                                 "speedup_decode": dense_decode_us / decode_us if decode_us else None,
                                  "kv_rows_retained_vs_dense": work["retained_fraction"]}
         del pipe
         torch.cuda.empty_cache()
@@ -547,7 +547,7 @@ def main():
         out["e2e"] = {"value": job_throughput(world, wl.batch, wl.L, e2e_prefill_ms), "unit": UNIT,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                       "prefill_ms": e2e_prefill_ms,
-                      "decode_us_per_step": st_e2e["decode"] * 1e3 / max(1, wl.decode_steps),
+                      "decode_us_per_step": st_e2e["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None,
                       "note": "pinned host buffers: K, V and the newest query copied in first; Q copied in and O copied "
                               "back in row ranges on two copy streams while tca_attn_prefill_rows computes the "
                               "ranges already present; decode tokens copied in, decode outputs copied back; the "
