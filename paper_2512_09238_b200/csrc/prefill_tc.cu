@@ -19,11 +19,13 @@
 // S columns and feeds the PV product straight from TMEM.  Shared memory: Q0 Q1 | 5-slot K/V ring.
 // Per tile the issuer runs  PV0(t) S0(t+1) PV1(t) S1(t+1)  so that S of one head is being
 // computed while the other head's softmax is in flight; the whole issuer warp executes the
-// loop and an elected lane's tcgen05 instructions take effect (see umma_ss_elect).  O stays in TMEM and is rescaled
-// lazily: only when a row maximum grew by more than 2^8 since the last rescale.  The softmax
-// arithmetic uses the packed fp32x2 forms (fma, add) and the three-input max, which halves its
-// issue slots.  CTAs are ordered unit-major so that the CTAs resident
-// at one time read the same one or two KV heads out of L2.
+// loop and an elected lane's tcgen05 instructions take effect (see umma_ss_elect).  O stays
+// in TMEM and is rescaled lazily: only when a row maximum grew by more than 2^8 since the last
+// rescale.  The softmax arithmetic uses the packed fp32x2 forms (fma, add) and the three-input
+// max, which halves its issue slots.  CTAs are ordered unit-major so that the CTAs resident
+// at one time read the same one or two KV heads out of L2.  With lse_out the kernel also
+// writes minus the log2 of each row's softmax denominator (used by the calibration pass), and
+// with O == nullptr it writes nothing else.
 //
 // Every mbarrier wait is bounded; a wait that gives up raises the status word of the
 // workspace, lets outstanding copies land, frees TMEM and returns.
