@@ -218,7 +218,7 @@ int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, c
  *                      bf16 only (TCA_ERR_UNSUPPORTED otherwise); colmean DEVICE [U][L] doubles;
  *                      ws DEVICE, tca_workspace_bytes(prm, L, TCA_OP_CALIB), word 0 is a status
  *                      word readable with tca_ws_status.  prm->block and prm->window are not
- *                      used.  Cost: two dense causal passes over Q K^T.
+ *                      used.  Cost: two dense causal passes over Q K^T (row log-sum-exps, then column sums).
  *   tca_calib_score    a[u] of Eq. 4 for the selection (idx, offsets_dev) that tca_select wrote
  *                      for one candidate, as a share of the sum over all candidates [0, m*b):
  *                      a 100 % budget scores exactly 1.  a_out DEVICE [U] doubles.

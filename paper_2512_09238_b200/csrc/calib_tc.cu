@@ -3,8 +3,8 @@
 //
 //   c[k] = 1/(G (L-k)) * sum_g sum_{j >= k} exp2(q_{g,j}.k_k * scale*log2e - lse2_{g,j})
 //
-// Pass 1 is the library's own prefill kernel run densely (window = L, empty global region)
-// with its per-row log-sum-exp written out instead of O.  Pass 2 (this file) keeps a tile of
+// Pass 1 computes the log-sum-exp of every query row (a tile of 128 queries stationary, the key
+// tiles before it streamed).  Pass 2 keeps a tile of
 // 128 keys stationary as the A operand and streams the query tiles at or after it as B:
 // S^T = K_tile Q_tile^T lands in TMEM with one key per lane, and the thread that owns the
 // lane exponentiates its 128 scores against the queries' log-sum-exps and adds them up.
@@ -33,11 +33,6 @@
 
 namespace tca {
 
-template <int D>
-int launch_prefill_tc(const tca_params*, const void*, const void*, const void*, int64_t, int64_t, int64_t,
-                      const tca_cache_desc*, void*, void*, cudaStream_t, float*, int64_t);
-size_t prefill_tc_ws_bytes(const tca_params* prm);
-
 namespace {
 
 constexpr int CT = 128;                  // keys per CTA and queries per tile
@@ -59,6 +54,211 @@ struct ColCfg {
 enum { CB_K = 0, CB_FULL = 1, CB_EMPTY = CB_FULL + kQRing, CB_S = CB_EMPTY + kQRing, CB_FREE = CB_S + 2,
        CN_BARS = CB_FREE + 2 };
 
+// ------------------------------------------------------------------ pass 1: row statistics
+// For every query row of every head: minus the log2 of the causal softmax denominator in the
+// units of the scaled scores, -(m + log2 sum_j exp2(s_j * scale - m)).  A tile of 128 queries
+// of two heads of the group stays in shared memory as the A operands of two chains; the key
+// tiles 0..qt stream through a ring and each feeds both chains (S_c = Q_c K_tile^T, one
+// query per TMEM lane).  The lane's thread keeps a running reference maximum (moved only when
+// a tile's maximum exceeds it by more than 2^8, the sum is rescaled then) and adds up the
+// exponentials.  No V, no P, no O: a chain's S buffer is free once its scores are in registers.
+template <int D>
+struct RowCfg {
+  static constexpr int NH = D / 64;
+  static constexpr int kTile = NH * kColHalfBytes;   // one Q or K tile
+  static constexpr int offQ = 0;                     // two Q tiles
+  static constexpr int offRing = 2 * kTile;
+  static constexpr int offBar = offRing + kQRing * kTile;
+  static constexpr int bytes = offBar + 256 + 1024;
+};
+
+enum { RB_Q = 0, RB_QFREE = 1, RB_FULL = 2, RB_EMPTY = RB_FULL + kQRing, RB_S = RB_EMPTY + kQRing, RB_FREE = RB_S + 2,
+       RN_BARS = RB_FREE + 2 };
+
+template <int D>
+__global__ void __launch_bounds__(kColThreads, 1)
+calib_rowstats_kernel(const CUtensorMap* __restrict__ maps, float* __restrict__ neg_lse, int64_t lse_stride, int64_t L,
+                      int n_q_heads, int n_kv_heads, float scale_log2e, int* __restrict__ status, int n_tiles) {
+  using Cfg = RowCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::offBar);
+  static_assert(RN_BARS <= 24, "barrier block");
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = n_q_heads / n_kv_heads;
+  const int u = int(blockIdx.x) / n_tiles;
+  const int qt = n_tiles - 1 - int(blockIdx.x) % n_tiles;   // the longest rows go first
+  const int seq = u / n_kv_heads, kvh = u % n_kv_heads;
+  const int head0 = seq * n_q_heads + kvh * G;
+  const int nk = qt + 1;                                     // key tiles 0 .. qt
+  const int n_pairs = (G + 1) / 2;
+
+  if (tid == 0) {
+    ptx::mbar_init(&bars[RB_Q], 1);
+    ptx::mbar_init(&bars[RB_QFREE], 1);
+    for (int i = 0; i < kQRing; ++i) {
+      ptx::mbar_init(&bars[RB_FULL + i], 1);
+      ptx::mbar_init(&bars[RB_EMPTY + i], 1);
+    }
+    for (int c = 0; c < 2; ++c) {
+      ptx::mbar_init(&bars[RB_S + c], 1);
+      ptx::mbar_init(&bars[RB_FREE + c], 128);
+    }
+    ptx::fence_barrier_init();
+    *abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
+  }
+  if (warp == 0) {
+    ptx::tmem_alloc(tmem_slot, 256);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (!*abort_flag) {
+    if (warp == 0) {
+      // ------------------------------------------------------------- TMA producer
+      if (lane == 0) {
+        int jj = 0;
+        bool ok = true;
+        for (int pair = 0; pair < n_pairs && ok; ++pair) {
+          const int nh = min(2, G - 2 * pair);
+          // the previous pair's products must have finished reading the Q tiles
+          if (pair > 0 && !ptx::mbar_wait(&bars[RB_QFREE], uint32_t(pair - 1) & 1u, abort_flag)) break;
+          ptx::mbar_arrive_expect_tx(&bars[RB_Q], uint32_t(nh * Cfg::kTile));
+          for (int c = 0; c < nh; ++c)
+            for (int half = 0; half < Cfg::NH; ++half)
+              ptx::tma_load_3d(smem + Cfg::offQ + c * Cfg::kTile + half * kColHalfBytes, &maps[0], half * 64, qt * CT,
+                               head0 + 2 * pair + c, &bars[RB_Q]);
+          for (int kt = 0; kt < nk; ++kt, ++jj) {
+            const int slot = jj % kQRing;
+            if (jj >= kQRing && !ptx::mbar_wait(&bars[RB_EMPTY + slot], uint32_t(jj / kQRing - 1) & 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            ptx::mbar_arrive_expect_tx(&bars[RB_FULL + slot], uint32_t(Cfg::kTile));
+            for (int half = 0; half < Cfg::NH; ++half)
+              ptx::tma_load_3d(smem + Cfg::offRing + slot * Cfg::kTile + half * kColHalfBytes, &maps[1], half * 64,
+                               kt * CT, u, &bars[RB_FULL + slot]);
+          }
+        }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------- MMA issuer (whole warp, elected lane)
+      {
+        constexpr uint32_t idesc = ptx::idesc_bf16(CT, CT, false);
+        const uint64_t dq = ptx::smem_desc_sw128(ptx::smem_u32(smem + Cfg::offQ), 16, 1024);      // queries as A
+        const uint64_t dk = ptx::smem_desc_sw128(ptx::smem_u32(smem + Cfg::offRing), 16, 1024);   // keys as B
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+          return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
+        };
+        int jj = 0;
+        uint32_t done[2] = {0u, 0u};
+        bool ok = true;
+        for (int pair = 0; pair < n_pairs && ok; ++pair) {
+          const int nh = min(2, G - 2 * pair);
+          ok = wait(&bars[RB_Q], uint32_t(pair) & 1u);
+          for (int kt = 0; kt < nk && ok; ++kt, ++jj) {
+            const int slot = jj % kQRing;
+            ok = wait(&bars[RB_FULL + slot], uint32_t(jj / kQRing) & 1u);
+            for (int c = 0; c < nh && ok; ++c) {
+              ok = done[c] == 0 || wait(&bars[RB_FREE + c], (done[c] - 1) & 1u);
+              if (!ok) break;
+              ptx::tc_fence_after();
+              const uint64_t a0 = dq + uint64_t(uint32_t(c * Cfg::kTile) >> 4);
+              const uint64_t b0 = dk + uint64_t(uint32_t(slot * Cfg::kTile) >> 4);
+              const uint32_t d = tmem_base + uint32_t(c) * CT;
+#pragma unroll
+              for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (uint32_t(kk >> 2) * kColHalfBytes + uint32_t(kk & 3) * 32u) >> 4;
+                ptx::umma_ss_elect(d, a0 + off, b0 + off, idesc, kk > 0);
+              }
+              ptx::umma_commit_elect(&bars[RB_S + c]);
+              ++done[c];
+            }
+            if (ok) ptx::umma_commit_elect(&bars[RB_EMPTY + slot]);
+          }
+          if (ok) ptx::umma_commit_elect(&bars[RB_QFREE]);
+        }
+      }
+    } else {
+      // ------------------------------------------------------------- one query row per thread
+      const int c = (warp - 2) >> 2;
+      const int quarter = warp & 3;
+      const int r = quarter * 32 + lane;
+      const int64_t i = int64_t(qt) * CT + r;
+      const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(c) * CT;
+      const uint64_t scale2 = ptx::pack2(scale_log2e, scale_log2e);
+      uint32_t done = 0;
+      bool ok = true;
+      for (int pair = 0; pair < n_pairs && ok; ++pair) {
+        if (2 * pair + c >= G) break;                        // uniform for the chain's four warps
+        float m_run = -INFINITY, m_used = -INFINITY, l = 0.f;
+        for (int kt = 0; kt < nk; ++kt) {
+          ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bars[RB_S + c], done & 1u, abort_flag));
+          if (!ok) break;
+          ++done;
+          ptx::tc_fence_after();
+          uint32_t v[CT];
+#pragma unroll
+          for (int q4 = 0; q4 < CT / 32; ++q4)
+            ptx::tmem_ld32(lane_addr + q4 * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[q4 * 32]));
+          ptx::tc_wait_ld();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(&bars[RB_FREE + c]);              // the scores are in registers
+          if (kt == qt) {                                     // diagonal tile: keys after the query are masked
+#pragma unroll
+            for (int k = 0; k < CT; ++k)
+              if (k > r) v[k] = 0xff800000u;
+          }
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int k = 0; k < CT; k += 8) {
+            mx4[0] = ptx::max3(mx4[0], __uint_as_float(v[k]), __uint_as_float(v[k + 1]));
+            mx4[1] = ptx::max3(mx4[1], __uint_as_float(v[k + 2]), __uint_as_float(v[k + 3]));
+            mx4[2] = ptx::max3(mx4[2], __uint_as_float(v[k + 4]), __uint_as_float(v[k + 5]));
+            mx4[3] = ptx::max3(mx4[3], __uint_as_float(v[k + 6]), __uint_as_float(v[k + 7]));
+          }
+          m_run = fmaxf(m_run, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2e);
+          if (m_run > m_used + 8.f) {                         // key 0 is visible to every row: m_run is finite
+            l *= (m_used == -INFINITY) ? 0.f : ptx::fast_exp2(m_used - m_run);
+            m_used = m_run;
+          }
+          const uint64_t neg_m2 = ptx::pack2(-m_used, -m_used);
+          uint64_t sum2[2] = {0ull, 0ull};
+#pragma unroll
+          for (int j = 0; j < CT / 2; ++j) {
+            float xl, xh;
+            ptx::unpack2(ptx::fma2(ptx::pack2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), scale2, neg_m2),
+                         xl, xh);
+            sum2[j & 1] = ptx::add2(sum2[j & 1], ptx::pack2(ptx::fast_exp2(xl), ptx::fast_exp2(xh)));
+          }
+          float s0, s1, s2, s3;
+          ptx::unpack2(sum2[0], s0, s1);
+          ptx::unpack2(sum2[1], s2, s3);
+          l += (s0 + s1) + (s2 + s3);
+        }
+        if (ok && i < L) neg_lse[size_t(head0 + 2 * pair + c) * lse_stride + size_t(i)] = -(m_used + log2f(l));
+      }
+    }
+  }
+
+  // ------------------------------------------------------------- teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (tid == 0) atomicExch(status, 1);
+    for (int k = 0; k < 64; ++k) __nanosleep(2000);  // let copies that are still in flight land
+    __syncthreads();
+  }
+  if (warp == 0) ptx::tmem_dealloc(tmem_base, 256);
+}
+
+// ------------------------------------------------------------------ pass 2: column sums
 template <int D>
 __global__ void __launch_bounds__(kColThreads, 1)
 calib_colsum_kernel(const CUtensorMap* __restrict__ maps, const float* __restrict__ neg_lse, int64_t lse_stride,
@@ -279,9 +479,7 @@ calib_score_kernel(const double* __restrict__ colmean, int64_t L, int64_t mb, co
 }
 
 struct CalibWs {
-  void* prefill;        // the dense pass's own workspace (status word + tensor maps)
-  int64_t* state;       // U x TCA_STATE_WORDS zero words: every unit with an empty global region
-  CUtensorMap* maps;    // Q and K for the column-sum kernel
+  CUtensorMap* maps;    // Q and K, shared by both passes
   float* neg_lse;       // [batch * n_q_heads][Lp]
   int64_t Lp;
   size_t bytes;
@@ -289,13 +487,8 @@ struct CalibWs {
 
 CalibWs calib_ws_layout(const tca_params* prm, int64_t L, void* ws) {
   CalibWs w;
-  const size_t U = size_t(prm->batch) * prm->n_kv_heads;
   char* p = static_cast<char*>(ws);
-  size_t off = 0;
-  w.prefill = p;
-  off += align_up(prefill_tc_ws_bytes(prm), 256);
-  w.state = reinterpret_cast<int64_t*>(p + off);
-  off += align_up(U * TCA_STATE_WORDS * sizeof(int64_t), 256);
+  size_t off = 256;     // word 0: status
   w.maps = reinterpret_cast<CUtensorMap*>(p + off);
   off += align_up(2 * sizeof(CUtensorMap), 256);
   w.Lp = (L + CT - 1) / CT * CT;
@@ -308,41 +501,31 @@ CalibWs calib_ws_layout(const tca_params* prm, int64_t L, void* ws) {
 template <int D>
 int launch_colmean(const tca_params* prm, const void* Q, const void* K, int64_t L, double* colmean, void* ws,
                    cudaStream_t stream) {
-  using Cfg = ColCfg<D>;
   const CalibWs w = calib_ws_layout(prm, L, ws);
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int64_t heads = int64_t(prm->batch) * prm->n_q_heads;
-  // status word, the dense pass's maps and the all-zero unit states
-  TCA_CHECK_CUDA(cudaMemsetAsync(ws, 0, size_t(reinterpret_cast<char*>(w.maps) - static_cast<char*>(ws)), stream));
-
-  // pass 1: dense causal attention (window = L, nothing in the global region), lse written, O not
-  tca_params dense = *prm;
-  dense.window = int(L);
-  std::vector<int64_t> zeros(size_t(U), 0);
-  tca_cache_desc desc = {};
-  desc.k = const_cast<void*>(K);
-  desc.v = const_cast<void*>(K);
-  desc.pos = reinterpret_cast<int32_t*>(w.state);
-  desc.state = w.state;
-  desc.rows_total = L;
-  desc.n_units = U;
-  desc.seg_start = zeros.data();
-  desc.n_global = zeros.data();
-  int st = launch_prefill_tc<D>(&dense, Q, K, K, L, 0, L, &desc, nullptr, w.prefill, stream, w.neg_lse, w.Lp);
-  if (st != TCA_OK) return st;
-
-  // pass 2: column sums
+  TCA_CHECK_CUDA(cudaMemsetAsync(ws, 0, 256, stream));   // status word
   CUtensorMap maps[2];
   if (!encode_map(&maps[0], Q, D, L, heads, L) || !encode_map(&maps[1], K, D, L, U, L)) return TCA_ERR_CUDA;
+  // pageable source: staged by the runtime before the call returns
   TCA_CHECK_CUDA(cudaMemcpyAsync(w.maps, maps, sizeof(maps), cudaMemcpyHostToDevice, stream));
-  auto kern = calib_colsum_kernel<D>;
-  TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::bytes));
   const int n_tiles = int((L + CT - 1) / CT);
   const int64_t n_ctas = int64_t(n_tiles) * U;
   if (n_ctas >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;
-  kern<<<unsigned(n_ctas), kColThreads, Cfg::bytes, stream>>>(
-      w.maps, w.neg_lse, w.Lp, L, prm->n_q_heads, prm->n_kv_heads, prm->sm_scale * 1.4426950408889634f, colmean,
-      static_cast<int*>(ws), n_tiles);
+  const float scale_log2e = prm->sm_scale * 1.4426950408889634f;
+
+  auto rows = calib_rowstats_kernel<D>;
+  TCA_CHECK_CUDA(cudaFuncSetAttribute(rows, cudaFuncAttributeMaxDynamicSharedMemorySize, RowCfg<D>::bytes));
+  rows<<<unsigned(n_ctas), kColThreads, RowCfg<D>::bytes, stream>>>(
+      w.maps, w.neg_lse, w.Lp, L, prm->n_q_heads, prm->n_kv_heads, scale_log2e, static_cast<int*>(ws), n_tiles);
+  int st = check_launch();
+  if (st != TCA_OK) return st;
+
+  auto cols = calib_colsum_kernel<D>;
+  TCA_CHECK_CUDA(cudaFuncSetAttribute(cols, cudaFuncAttributeMaxDynamicSharedMemorySize, ColCfg<D>::bytes));
+  cols<<<unsigned(n_ctas), kColThreads, ColCfg<D>::bytes, stream>>>(
+      w.maps, w.neg_lse, w.Lp, L, prm->n_q_heads, prm->n_kv_heads, scale_log2e, colmean, static_cast<int*>(ws),
+      n_tiles);
   return check_launch();
 }
 

@@ -9,7 +9,7 @@ int launch_prefill_simt(const tca_params*, const void*, const void*, const void*
                         const tca_cache_desc*, void*, cudaStream_t);
 template <int D>
 int launch_prefill_tc(const tca_params*, const void*, const void*, const void*, int64_t, int64_t, int64_t,
-                      const tca_cache_desc*, void*, void*, cudaStream_t, float*, int64_t);
+                      const tca_cache_desc*, void*, void*, cudaStream_t);
 }  // namespace tca
 
 using namespace tca;
@@ -41,8 +41,8 @@ extern "C" int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const
     return launch_prefill_simt<__nv_bfloat16, 64>(prm, Q, K, V, L, row_begin, row_end, c, O, s);
   }
   TCA_CHECK_ARG(c->seg_start && c->n_global);
-  if (prm->head_dim == 128) return launch_prefill_tc<128>(prm, Q, K, V, L, row_begin, row_end, c, O, ws, s, nullptr, 0);
-  return launch_prefill_tc<64>(prm, Q, K, V, L, row_begin, row_end, c, O, ws, s, nullptr, 0);
+  if (prm->head_dim == 128) return launch_prefill_tc<128>(prm, Q, K, V, L, row_begin, row_end, c, O, ws, s);
+  return launch_prefill_tc<64>(prm, Q, K, V, L, row_begin, row_end, c, O, ws, s);
 }
 
 extern "C" int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,

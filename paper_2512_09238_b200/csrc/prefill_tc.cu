@@ -23,9 +23,7 @@
 // in TMEM and is rescaled lazily: only when a row maximum grew by more than 2^8 since the last
 // rescale.  The softmax arithmetic uses the packed fp32x2 forms (fma, add) and the three-input
 // max, which halves its issue slots.  CTAs are ordered unit-major so that the CTAs resident
-// at one time read the same one or two KV heads out of L2.  With lse_out the kernel also
-// writes minus the log2 of each row's softmax denominator (used by the calibration pass), and
-// with O == nullptr it writes nothing else.
+// at one time read the same one or two KV heads out of L2.
 //
 // Every mbarrier wait is bounded; a wait that gives up raises the status word of the
 // workspace, lets outstanding copies land, frees TMEM and returns.
@@ -87,7 +85,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restrict__ pos,
                   const int64_t* __restrict__ state, int64_t L, int n_q_heads, int n_kv_heads, int window,
                   int64_t mb, float scale_log2e, __nv_bfloat16* __restrict__ O, int* __restrict__ status,
-                  int n_qtiles, int pairs_per_unit, int tile0, float* __restrict__ lse_out, int64_t lse_stride) {
+                  int n_qtiles, int pairs_per_unit, int tile0) {
   using Cfg = TcCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -342,12 +340,9 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
         if (ok) {
           ptx::tc_fence_after();
           const float inv = 1.f / l;
-          // minus the log2 of the row's softmax denominator, in the units of the scaled scores: the
-          // calibration pass adds it to a scaled score to get the log2 of a probability
-          if (lse_out != nullptr && i <= i_last) lse_out[size_t(hq0 + h) * lse_stride + size_t(i)] = -(m_used + log2f(l));
           __nv_bfloat16* orow = O + (size_t(hq0 + h) * L + size_t(i)) * D;
 #pragma unroll 1
-          for (int c = 0; c < D / 32 && O != nullptr; ++c) {
+          for (int c = 0; c < D / 32; ++c) {
             uint32_t v[32];
             ptx::tmem_ld32(lane_addr + Cfg::colO(h) + c * 32, v);
             ptx::tc_wait_ld();
@@ -390,7 +385,7 @@ size_t prefill_tc_ws_bytes(const tca_params* prm) {
 template <int D>
 int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
                       int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O, void* ws,
-                      cudaStream_t stream, float* lse_out, int64_t lse_stride) {
+                      cudaStream_t stream) {
   using Cfg = TcCfg<D>;
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int G = prm->n_q_heads / prm->n_kv_heads;
@@ -418,14 +413,13 @@ int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const
   const int64_t mb = num_blocks(prm, L) * prm->block;
   kern<<<unsigned(n_ctas), kThreads, Cfg::bytes, stream>>>(
       maps_dev, c->pos, c->state, L, prm->n_q_heads, prm->n_kv_heads, prm->window, mb,
-      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs, tile0, lse_out,
-      lse_stride);
+      prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs, tile0);
   return check_launch();
 }
 
 template int launch_prefill_tc<64>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
-                                   int64_t, const tca_cache_desc*, void*, void*, cudaStream_t, float*, int64_t);
+                                   int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
 template int launch_prefill_tc<128>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
-                                    int64_t, const tca_cache_desc*, void*, void*, cudaStream_t, float*, int64_t);
+                                    int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
 
 }  // namespace tca
