@@ -267,6 +267,10 @@ class Pipeline:
         self.h_Od.copy_(self.Od, non_blocking=True)
         if mark: self._ev("t_decode")
 
+    def step_ms(self):
+        """Milliseconds of every marked step (begin of the step to the end of its decode loop)."""
+        return [x.elapsed_time(y) for x, y in zip(self.ev["t_begin"], self.ev["t_decode"])]
+
     def stage_ms(self):
         """Mean milliseconds per stage over the marked steps."""
         names = ["t_begin", "t0", "t_score", "t_select", "t_compact", "t_prefill", "t_prefill_io", "t_decode"]
@@ -374,7 +378,15 @@ def time_oracle(wl, data, p, budget_s: float = 20.0):
         n_done += 1
     t_row = (time.perf_counter() - t1) / max(1, n_done)
     full = t_select * wl.batch * wl.n_kv_heads + t_row * L * wl.batch * wl.n_q_heads
+    # one decode step of the oracle: one query of one head over the retained rows, times the heads
+    T = res["T"]
+    Kt, Vt = K[T], V[T]
+    t2 = time.perf_counter()
+    for _ in range(3):
+        O.attention_over_set(Q[L - 1], Kt, Vt, scale)
+    t_dec = (time.perf_counter() - t2) / 3 * wl.batch * wl.n_q_heads
     return {"value": wl.batch * L / full, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "decode_us_per_step": t_dec * 1e6,
             "sample": f"select of 1 of {wl.batch * wl.n_kv_heads} KV heads at L={L} ({t_select:.2f} s) + "
                       f"{n_done} query rows of 1 head ({t_row * 1e3:.1f} ms/row); prefill time extrapolated "
                       f"to {wl.batch * wl.n_q_heads} heads x {L} rows"}
@@ -384,8 +396,8 @@ def time_oracle(wl, data, p, budget_s: float = 20.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="config4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--length", type=int, default=0, help="override L (smaller runs for profiling)")
@@ -478,6 +490,8 @@ def main():
         clocks = sampler.stop()
         ms = e0.elapsed_time(e1)
         stages = pipe.stage_ms()
+        per_step = pipe.step_ms()
+        stages["step_median"], stages["step_min"] = float(np.median(per_step)), float(np.min(per_step))
         red = reduce_max([ms] + [stages[k] for k in sorted(stages)], world, device="cuda")
         ms, stages = red[0], dict(zip(sorted(stages), red[1:]))
         return ms / args.steps, stages, clocks
@@ -492,6 +506,7 @@ def main():
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": config,
+           "ms_per_step_median": stages["step_median"], "ms_per_step_min": stages["step_min"],
            "decode_us_per_step": decode_us, "prefill_ms": prefill_ms, "clocks": clocks,
            "gpu_launches": pipe.launches_per_step * args.steps}
 
