@@ -28,8 +28,9 @@ notes with its justification):
     that Psi has exactly m entries;
   * ties inside Top(t; B) go to the lower token index;
   * decoding: the block that leaves the window is the one compressed;
-  * Algorithm 1: column means over the causally visible rows; the aggregated score is taken
-    as a share of its value at a 100 % budget; no valid candidate => the last candidate.
+  * Algorithm 1: column means over the causally visible rows; the aggregated score is the
+    share of the summed column means that the retained set (selected tokens and the always-kept
+    tail, the S_total of Section 4.3) holds; no valid candidate => the last candidate.
 
 Parity pins (tests/test_oracle_pins.py): dense causal attention by an independent
 brute force at 100 % budget and at w >= L; masked attention against an independently
@@ -285,15 +286,20 @@ def attention_column_means(Q: np.ndarray, K: np.ndarray, sm_scale: float) -> np.
 
 
 def aggregated_score(S: np.ndarray, c: np.ndarray, n_candidates: int) -> float:
-    """a_i of Eq. 4 for the selected set S, as a share of what selecting every candidate gives.
+    """a_i of Eq. 4 for the selected set S: the share of the aggregated score that is retained.
 
-    Eq. 4 is the plain sum of c over S.  The threshold tau of Algorithm 1 is "a share of the
-    aggregated attention mass", and the plain sum is not bounded by 1 (it depends on L and on how
-    local the head is), so the sum is divided by its value for S = all candidates [0, m*b): the
-    100 % configuration then scores exactly 1.
+    Eq. 4 is the sum of c over the selected tokens.  Algorithm 1 compares it with a threshold
+    tau in [0, 1] that the text calls a share "of the aggregated attention mass", and Section 4.3
+    argues from "retained mass >= tau" to "dropped mass <= 1 - tau" with the retained set being
+    the global subset AND the local subset.  So the sum runs over everything the method keeps,
+    T = S union [n_candidates, L) (the always-kept tail is the local subset of the newest
+    query), and is divided by the sum over all L tokens: keeping everything scores exactly 1,
+    and 1 - a_i is the share of the score that is dropped.
     """
-    total = float(np.sum(c[:n_candidates]))
-    return float(np.sum(c[np.asarray(S, dtype=np.int64)])) / total if total > 0.0 else 1.0
+    c = np.asarray(c, dtype=np.float64)
+    total = float(np.sum(c))
+    kept = float(np.sum(c[np.asarray(S, dtype=np.int64)])) + float(np.sum(c[n_candidates:]))
+    return kept / total if total > 0.0 else 1.0
 
 
 def calibrate_head(Q: np.ndarray, K: np.ndarray, candidates: np.ndarray, b: int, w: int, alpha: float,

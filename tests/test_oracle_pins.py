@@ -367,6 +367,9 @@ def test_candidate_grid_closed_forms(golden):
     # budgets grow monotonically from efficiency- to accuracy-oriented
     mean_keep = C @ O.retain_counts(b)
     assert np.all(np.diff(mean_keep) > 0)
+    # mean tokens kept per 128-token block for the 14 candidates, to the two decimals stored
+    assert len(g["mean_retention"]) == M
+    np.testing.assert_allclose(mean_keep, g["mean_retention"], atol=0.0051, rtol=0)   # half a unit of the last digit
 
 
 # ----------------------------------------------------------------------------- Algorithm 1 / Eq. 4
@@ -400,11 +403,26 @@ def test_column_means_against_a_masked_dense_matrix():
     assert float(np.sum(c1 * (L - np.arange(L)))) == pytest.approx(L, rel=1e-12)
 
 
-def test_aggregated_score_is_a_share_of_the_full_selection():
-    c = np.array([0.5, 0.25, 0.125, 0.125, 9.0, 9.0])      # 4 candidates, 2 always-kept tail tokens
+def test_aggregated_score_is_the_retained_share_of_all_column_means():
+    """4 candidates and 2 always-kept tail tokens, values chosen so that the plain sum of Eq. 4
+    (0.625), a share of the candidates only (0.625 / 1.125), a share of everything without the
+    tail in the numerator (0.625 / 4.125) and the retained share (3.625 / 4.125) all differ."""
+    c = np.array([0.5, 0.25, 0.125, 0.25, 2.0, 1.0])
+    assert O.aggregated_score(np.array([0, 2]), c, 4) == pytest.approx(3.625 / 4.125, rel=1e-15)
     assert O.aggregated_score(np.arange(4), c, 4) == pytest.approx(1.0, rel=1e-15)
-    assert O.aggregated_score(np.array([0, 2]), c, 4) == pytest.approx(0.625, rel=1e-15)
-    assert O.aggregated_score(np.array([], dtype=np.int64), c, 4) == 0.0
+    assert O.aggregated_score(np.array([], dtype=np.int64), c, 4) == pytest.approx(3.0 / 4.125, rel=1e-15)
+    # no tail at all: the share of the candidates
+    assert O.aggregated_score(np.array([1]), c[:4], 4) == pytest.approx(0.25 / 1.125, rel=1e-15)
+
+
+def test_aggregated_score_is_one_minus_the_dropped_share():
+    """Section 4.3 reads the threshold as a bound on what is dropped: a_i = 1 - (column means of
+    the tokens that are neither selected nor in the tail) / (all column means)."""
+    rng = _rng(23)
+    c = rng.random(40)
+    S = np.array([0, 3, 4, 17, 22])
+    dropped = np.setdiff1d(np.arange(32), S)
+    assert O.aggregated_score(S, c, 32) == pytest.approx(1.0 - c[dropped].sum() / c.sum(), rel=1e-13)
 
 
 def test_calibration_picks_the_sparsest_candidate_that_reaches_tau():
@@ -426,11 +444,12 @@ def test_calibration_picks_the_sparsest_candidate_that_reaches_tau():
     assert list(sizes) == [2, 4, 8]
     assert a[2] == pytest.approx(1.0, rel=1e-12) and np.all(np.diff(a) > 0)
     assert a[0] > 0.9 and choice == 0
-    # what candidate 0 selects is those two tokens, and a_0 is their share of the column means
+    # what candidate 0 selects is those two tokens; a_0 is the share of the column means that
+    # they and the always-kept tail [8, 12) hold
     r = O.select_head(Q[:, L - 1], K, cands[0], b, w, 0.5, 1.0)
     assert list(r["S"]) == [1, 6]
     c = O.attention_column_means(Q, K, 1.0)
-    assert a[0] == pytest.approx((c[1] + c[6]) / c[:8].sum(), rel=1e-12)
+    assert a[0] == pytest.approx((c[1] + c[6] + c[8:].sum()) / c.sum(), rel=1e-12)
     choice_hi, _, _ = O.calibrate_head(Q, K, cands, b, w, 0.5, 0.9999, 1.0)
     assert choice_hi == 2
     # a threshold nothing reaches falls back to the last candidate; equal sizes go to the lower index
