@@ -180,7 +180,7 @@ class Pipeline:
             self.row_ranges = list(zip(cuts[:-1], cuts[1:]))[::-1]
             self.ws_rows = [B.alloc_workspace(self.prm, wl.L, B.TCA_OP_PREFILL) for _ in self.row_ranges]
             self.h_Od = torch.empty_like(self.h_qd).pin_memory()
-        self.launches_per_step = 2 + 3 + 1 + 1 + wl.decode_steps * 3
+        self.launches_per_step = 2 + 3 + 1 + 1 + wl.decode_steps * 3   # score 2, select 3, compact, prefill; append + split + combine per step
         self.ev = {}
 
     def _ev(self, name):
@@ -498,6 +498,7 @@ def main():
 
     ms_step, stages, clocks = timed(host_io=False)
     assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    assert B.tca_ws_status(pipe.ws_decode) == B.TCA_OK     # no decode step timed on stale partials
     work = pipe.algorithmic_work()
     prefill_ms = stages["score"] + stages["select"] + stages["compact"] + stages["prefill"]
     value = job_throughput(world, wl.batch, wl.L, prefill_ms)

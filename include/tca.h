@@ -5,14 +5,24 @@
  *
  * Conventions
  *   - Every pointer is labelled HOST or DEVICE.  All device buffers (inputs, outputs,
- *     cache, workspace) are allocated and freed by the caller; the library allocates no
- *     device memory and keeps no global state.
+ *     cache, workspace) are allocated and freed by the caller; the library calls no
+ *     allocator.  What it keeps between calls is limited to: the built-in scratch array of
+ *     tca_attn_decode_static (and its per-device address), a small cache of encoded TMA
+ *     tensor maps keyed by buffer address and shape, and per-device constants (SM count).
  *   - Tensors are row-major with the head dimension contiguous:
  *       Q [batch, n_q_heads, L, head_dim]      K, V [batch, n_kv_heads, L, head_dim]
  *     A "unit" is one (sequence, KV head) pair, u = seq * n_kv_heads + kv_head; the G =
  *     n_q_heads / n_kv_heads query heads kv_head*G .. kv_head*G+G-1 share it.
  *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*); no call
- *     synchronises the host.  Outputs are valid once the stream has been synchronised.
+ *     synchronises the host except the three that read a status back (tca_ws_status,
+ *     tca_cache_status, tca_decode_static_status).  Outputs are valid once the stream has
+ *     been synchronised.
+ *   - Status words.  Word 0 of the prefill, decode, select and calibration workspaces is a
+ *     STICKY status word: zero it once after allocating (a zero-filled workspace is fine); a
+ *     kernel sets it when one of its bounded device-side waits gives up (or, in the
+ *     range-checked build, when an index is out of range) and nothing in the library clears
+ *     it.  While it is set, the tensor-core kernels return at once without computing.  After
+ *     a non-zero status, zero the whole workspace before using it again.
  *   - Return value: TCA_OK or a negative error.  Argument errors are detected on the
  *     host before anything is launched and leave every output untouched.  Unsupported
  *     shapes return TCA_ERR_UNSUPPORTED; nothing ever falls back to the CPU.
@@ -38,7 +48,8 @@ enum {
   TCA_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                   */
   TCA_ERR_TIMEOUT = -5,     /* a bounded device-side wait gave up (see tca_ws_status)   */
   TCA_ERR_CAPACITY = -6,    /* a cache region would overflow                            */
-  TCA_ERR_SCRATCH_LIMIT = -7 /* problem larger than the built-in scratch of a *_static call */
+  TCA_ERR_SCRATCH_LIMIT = -7, /* problem larger than the built-in scratch of a *_static call */
+  TCA_ERR_BOUNDS = -8        /* range-checked build only: an index or offset was out of range  */
 };
 
 enum { TCA_F32 = 0, TCA_BF16 = 1 };
@@ -59,7 +70,7 @@ typedef struct tca_params {
   int32_t n_kv_heads;
   int32_t head_dim;   /* d_h: 64 or 128                                                 */
   int32_t block;      /* b: power of two, 1..128 (Section 4.1)                          */
-  int32_t window;     /* w >= 0: local subset size (Section 4)                          */
+  int32_t window;     /* w >= 0: local subset size (Section 4); the prefill needs w >= 1 */
   float alpha;        /* balance of Eq. 6, in [0, 1]                                    */
   float sm_scale;     /* 1/sqrt(d_h) of Eqs. 2 and 5                                    */
   int32_t dtype;      /* TCA_F32 or TCA_BF16: element type of Q, K, V, O and the cache  */
@@ -160,9 +171,12 @@ int tca_select(const tca_params* prm, const double* logscore, int64_t L,
                const int32_t* n_k, int32_t nK, int32_t* idx, const int64_t* offsets_dev,
                double* h_out, int32_t* t_out, void* ws, size_t ws_bytes, void* stream);
 
-/* Upload the host mirror of `cache` (seg_start, global_cap, n_global, tail_head, n_tail,
- * seq_len, t_keep) into cache->state and zero-fill cache->k and cache->v (rows that are
- * not in use must hold finite values).  Call once after filling the descriptor. */
+/* REQUIRED once after filling the descriptor and before any other call that takes it:
+ * uploads the host mirror of `cache` (seg_start, global_cap, n_global, tail_head, n_tail,
+ * seq_len, t_keep) into cache->state and zero-fills cache->k and cache->v.  The zero-fill is
+ * not optional: the attention kernels multiply rows that are not in use by an exactly zero
+ * weight, which cancels only finite values, so a cache that skips this call can turn
+ * uninitialised memory into NaNs in the output without any error being reported. */
 int tca_cache_init(const tca_params* prm, tca_cache_desc* cache, void* stream);
 
 /*
@@ -183,8 +197,10 @@ int tca_compact_kv(const tca_params* prm, const void* K, const void* V, int64_t 
  * attends to {j <= i : j in S or j >= c_i}, c_i = min(max(0, i - w + 1), m*b): its own
  * last w keys (read from K, V) plus the selected keys before them (read from the cache's
  * global region); every key is counted once.  O has the shape of Q.
- *   ws   DEVICE workspace, tca_workspace_bytes(prm, L, TCA_OP_PREFILL); word 0 is a status
- *        word readable with tca_ws_status.
+ *   ws   DEVICE workspace, tca_workspace_bytes(prm, L, TCA_OP_PREFILL); word 0 is the sticky
+ *        status word (see Conventions), readable with tca_ws_status.
+ * prm->window must be >= 1 (TCA_ERR_UNSUPPORTED otherwise): with w = 0 a query that is not
+ * itself selected would attend to nothing, and Eq. 2 has no value for an empty key set.
  */
 int tca_attn_prefill(const tca_params* prm, const void* Q, const void* K, const void* V,
                      int64_t L, const tca_cache_desc* cache, void* O,
@@ -220,8 +236,11 @@ int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, c
  *                      word readable with tca_ws_status.  prm->block and prm->window are not
  *                      used.  Cost: two dense causal passes over Q K^T (row log-sum-exps, then column sums).
  *   tca_calib_score    a[u] of Eq. 4 for the selection (idx, offsets_dev) that tca_select wrote
- *                      for one candidate, as a share of the sum over all candidates [0, m*b):
- *                      a 100 % budget scores exactly 1.  a_out DEVICE [U] doubles.
+ *                      for one candidate: the column means summed over everything the method
+ *                      retains (the selected tokens and the always-kept tail [m*b, L), the
+ *                      S_total of Section 4.3), as a share of the sum over all L tokens.  A
+ *                      100 % budget scores exactly 1 and 1 - a is the share that is dropped.
+ *                      a_out DEVICE [U] doubles.
  *   tca_calib_choose   HOST: the index of the candidate with the fewest selected tokens among
  *                      those with a[i] >= tau (the lowest index on a tie); if none reaches tau,
  *                      n_candidates - 1.  a, sizes HOST arrays of n_candidates entries.
@@ -247,9 +266,11 @@ int tca_calib_candidates(int block, int n_candidates, double sigma, double* p_ou
  * One decode step, Eq. 2 with a single query per head over the whole retained cache
  * (global region + tail ring) of its KV head.
  *   q  DEVICE [batch, n_q_heads, head_dim]     O  DEVICE out, same shape
- *   ws DEVICE workspace, tca_workspace_bytes(prm, cache->rows_total, TCA_OP_DECODE).  Its
- *      first word is a sticky error flag (tca_ws_status): zero it once after allocating;
- *      a kernel sets it if one of its bounded waits gave up, and never clears it.
+ *   ws DEVICE workspace, tca_workspace_bytes(prm, cache->rows_total, TCA_OP_DECODE), zeroed
+ *      once after allocating.  Word 0 is the sticky status word (tca_ws_status).  Every CTA
+ *      leaves a partial result for its slice of a unit's rows in the workspace and a second,
+ *      small kernel merges each unit's partials in slice order.  Calls that share a workspace
+ *      must not overlap on the GPU.
  */
 int tca_attn_decode(const tca_params* prm, const void* q, const tca_cache_desc* cache,
                     void* O, void* ws, size_t ws_bytes, void* stream);
@@ -284,25 +305,52 @@ int tca_cache_append(const tca_params* prm, tca_cache_desc* cache, const void* k
  *
  *   q, cache, O, stream   as for tca_attn_decode; inputs and outputs still belong to the
  *                         caller.
- *   Limit   the partials need (rows_total / 256 + 2 * n_units + 1) * G * (head_dim + 2) * 4
- *           bytes; a cache for which that exceeds the array (about 2 million rows at
- *           G = 4, head_dim = 128) is refused with TCA_ERR_SCRATCH_LIMIT and nothing is
- *           launched.  Use tca_attn_decode with a workspace of your own for larger caches.
+ *   Limit   the call needs what tca_workspace_bytes(prm, rows_total, TCA_OP_DECODE) reports:
+ *             256 + roundup256((rows_total / 256 + 2 * n_units + 1) * G * (head_dim + 2) * 4)
+ *           bytes (roundup256 = up to a multiple of 256; rows_total / 256 rounds down).  A
+ *           cache for which that exceeds the array (about 2 million rows at G = 4,
+ *           head_dim = 128) is refused with TCA_ERR_SCRATCH_LIMIT and nothing is launched.
+ *           Use tca_attn_decode with a workspace of your own for larger caches.
  *   Set-up  the first call on each device looks up the array's device address (with that
  *           device current) and remembers it; make that first call outside any stream
  *           capture.
  *   Sharing every call on a device uses the same array, which keeps the previous call's
- *           contents.  Nothing in it has to start at zero (each partial is written before
- *           it is read), but two calls that overlap on the GPU (different streams, or
- *           different threads without ordering) race on it and corrupt each other:
- *           serialise them.
+ *           contents.  Nothing in it has to be cleared by the caller: the status word is zero
+ *           when the library is loaded and tca_decode_static_status clears it after reporting
+ *           a failure, and each partial is written before it is read.  Two calls that overlap
+ *           on the GPU (different streams, or different threads without ordering) race on
+ *           the array and corrupt each other: serialise them.
+ *   Errors  the status word of this variant lives inside the array, where tca_ws_status
+ *           cannot reach it; tca_decode_static_status reads it instead.
  */
 int tca_attn_decode_static(const tca_params* prm, const void* q, const tca_cache_desc* cache,
                            void* O, void* stream);
 
-/* Synchronise `stream` and read the status word a kernel left at the start of a
- * workspace: TCA_OK, or TCA_ERR_TIMEOUT if a bounded wait inside the kernel expired. */
+/* Synchronise `stream`, then report whether a bounded wait gave up in a tca_attn_decode_static
+ * call on the current device since the last time this was asked: TCA_OK, or TCA_ERR_TIMEOUT (the
+ * outputs of the calls since then are not valid).  After TCA_ERR_TIMEOUT the status word in the
+ * array has been cleared and the entry point can be used again.  Performs no allocation.  (No
+ * counterpart in the paper.) */
+int tca_decode_static_status(void* stream);
+
+/* Synchronise `stream` and read the sticky status word at the start of a workspace: TCA_OK,
+ * TCA_ERR_TIMEOUT if a bounded wait inside a kernel gave up, or (range-checked build)
+ * TCA_ERR_BOUNDS if a kernel met an index or offset outside its range and skipped the access. */
 int tca_ws_status(const void* ws, void* stream);
+
+/*
+ * Self-test of the abort path that every bounded device-side wait shares.  One small CTA with the
+ * roles of the attention kernels (a warp that holds tensor memory, one waiter with a time limit,
+ * waiters that watch the CTA's abort flag) waits on a barrier at which nothing ever arrives.  After
+ * limit_ns the limited wait gives up, the other waiters leave on the flag, the CTA sets word 0 of
+ * `ws` exactly as the production kernels do, frees its tensor memory and returns.  Nothing traps
+ * and nothing waits without a limit.  Afterwards tca_ws_status(ws) is TCA_ERR_TIMEOUT.
+ *   ws             DEVICE, at least 256 bytes, 256-byte aligned, word 0 zero on entry
+ *   limit_ns       1000 .. 100000000 (1 us .. 100 ms), else TCA_ERR_INVALID_ARG
+ *   waited_ns_dev  DEVICE out, optional: how long the limited wait actually lasted
+ * (No counterpart in the paper: test support for the library's error handling.)
+ */
+int tca_selftest_wait_expiry(void* ws, uint64_t limit_ns, uint64_t* waited_ns_dev, void* stream);
 
 #ifdef __cplusplus
 }

@@ -57,7 +57,8 @@ __all__ = [
     "budget_map", "mean_retain_floor", "rank_blocks", "block_requirement",
     "select_tokens", "retained_set", "select_head", "visible_mask_row",
     "attention_rows", "attention_over_set", "candidate_grid", "DecodeCache",
-    "dropped_mass", "attention_column_means", "aggregated_score", "calibrate_head",
+    "dropped_mass", "attention_column_means", "attention_column_means_at", "aggregated_score",
+    "calibrate_head",
 ]
 
 
@@ -283,6 +284,37 @@ def attention_column_means(Q: np.ndarray, K: np.ndarray, sm_scale: float) -> np.
             e = np.exp(x)
             col[:j + 1] += e / e.sum()
     return col / (G * (L - np.arange(L, dtype=np.float64)))
+
+
+def attention_column_means_at(Q: np.ndarray, K: np.ndarray, sm_scale: float, cols: Sequence[int],
+                              rows_per_step: int = 512) -> np.ndarray:
+    """attention_column_means for the chosen columns only, for sequences too long to afford all.
+
+    The same definition: c[k] = (1 / (L - k)) * sum_{j >= k} A[j, k], averaged over the G query
+    heads, with A[j, :] the softmax of row j over its visible keys 0..j.  Rows are taken
+    `rows_per_step` at a time only so that the logits of a step fit in memory (one matrix product
+    per step instead of one product per row); every row's softmax is still normalised over all of
+    its visible keys.  Returns [len(cols)].
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    if Q.ndim == 2:
+        Q = Q[None]
+    G, L, _ = Q.shape
+    cols = np.asarray(cols, dtype=np.int64)
+    total = np.zeros(len(cols), dtype=np.float64)
+    for g in range(G):
+        for j0 in range(0, L, rows_per_step):
+            j1 = min(L, j0 + rows_per_step)
+            x = (Q[g, j0:j1] @ K[:j1].T) * sm_scale                  # rows j0..j1-1, keys 0..j1-1
+            key = np.arange(j1)[None, :]
+            row = np.arange(j0, j1)[:, None]
+            x = np.where(key <= row, x, -np.inf)                      # causal: row j sees keys <= j
+            lse = _logsumexp(x, axis=1)
+            seen = cols < j1
+            a = np.exp(x[:, cols[seen]] - lse[:, None])               # masked entries are exactly 0
+            total[seen] += a.sum(axis=0)
+    return total / (G * (L - cols.astype(np.float64)))
 
 
 def aggregated_score(S: np.ndarray, c: np.ndarray, n_candidates: int) -> float:

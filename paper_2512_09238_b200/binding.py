@@ -19,7 +19,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libtca.so")
 
 TCA_OK, TCA_ERR_INVALID_ARG, TCA_ERR_UNSUPPORTED, TCA_ERR_WORKSPACE = 0, -1, -2, -3
-TCA_ERR_CUDA, TCA_ERR_TIMEOUT, TCA_ERR_CAPACITY, TCA_ERR_SCRATCH_LIMIT = -4, -5, -6, -7
+TCA_ERR_CUDA, TCA_ERR_TIMEOUT, TCA_ERR_CAPACITY, TCA_ERR_SCRATCH_LIMIT, TCA_ERR_BOUNDS = -4, -5, -6, -7, -8
 TCA_DECODE_STATIC_SCRATCH_BYTES = 16 << 20
 TCA_F32, TCA_BF16 = 0, 1
 TCA_FLAG_PREFILL_SIMT = 1
@@ -31,6 +31,7 @@ EXPORTS = (
     "tca_select", "tca_cache_init", "tca_compact_kv", "tca_attn_prefill", "tca_attn_decode",
     "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
     "tca_calib_colmean", "tca_calib_score", "tca_calib_choose", "tca_calib_candidates",
+    "tca_decode_static_status", "tca_selftest_wait_expiry",
 )
 
 
@@ -90,6 +91,8 @@ def lib() -> C.CDLL:
         L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
         L.tca_ws_status.argtypes = [vp, vp]
         L.tca_attn_decode_static.argtypes = [P, vp, D, vp, vp]
+        L.tca_decode_static_status.argtypes = [vp]
+        L.tca_selftest_wait_expiry.argtypes = [vp, C.c_uint64, vp, vp]
         for name in EXPORTS:
             if name not in ("tca_strerror", "tca_workspace_bytes"):
                 getattr(L, name).restype = C.c_int
@@ -214,6 +217,19 @@ def tca_attn_decode_static(prm, q, cache: "Cache", O, stream=None) -> None:
     loop).  Calls share that array: do not let two of them overlap on the GPU."""
     _check(lib().tca_attn_decode_static(C.byref(prm), _dev(q), C.byref(cache.desc), _dev(O), _stream(stream)),
            "tca_attn_decode_static")
+
+
+def tca_decode_static_status(stream=None) -> int:
+    """TCA_OK, or TCA_ERR_TIMEOUT if a bounded wait gave up inside a tca_attn_decode_static call on
+    this device since the last query (the array's status word and counters are then cleared)."""
+    return lib().tca_decode_static_status(_stream(stream))
+
+
+def tca_selftest_wait_expiry(ws, limit_ns: int, waited_ns=None, stream=None) -> None:
+    """Makes one bounded device-side wait run out after limit_ns and leave through the kernels'
+    abort path; afterwards tca_ws_status(ws) is TCA_ERR_TIMEOUT."""
+    _check(lib().tca_selftest_wait_expiry(_dev(ws), int(limit_ns), _dev(waited_ns), _stream(stream)),
+           "tca_selftest_wait_expiry")
 
 
 def tca_cache_append(prm, cache: "Cache", k_new, v_new, q_cur, stream=None) -> None:

@@ -57,8 +57,8 @@ DecodeWs decode_ws_layout(const tca_params* prm, int64_t rows_total, int64_t n_u
   // slices are at least kDecodeChunkRows long, plus one short slice per unit
   w.n_chunks_max = rows_total / kDecodeChunkRows + 2 * n_units + 1;
   w.status = reinterpret_cast<int*>(ws);
-  w.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + 256);
-  w.bytes = 256 + align_up(size_t(w.n_chunks_max) * G * (prm->head_dim + 2) * sizeof(float), 256);
+  w.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + kDecodeHeaderBytes);
+  w.bytes = kDecodeHeaderBytes + align_up(size_t(w.n_chunks_max) * G * (prm->head_dim + 2) * sizeof(float), 256);
   return w;
 }
 
@@ -78,6 +78,7 @@ const char* tca_strerror(int status) {
     case TCA_ERR_TIMEOUT: return "device-side wait timed out";
     case TCA_ERR_CAPACITY: return "cache capacity exceeded";
     case TCA_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the static entry point";
+    case TCA_ERR_BOUNDS: return "index or offset out of range (range-checked build)";
     default: return "unknown status";
   }
 }
@@ -191,7 +192,7 @@ int tca_ws_status(const void* ws, void* stream) {
   TCA_CHECK_CUDA(cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost,
                                  static_cast<cudaStream_t>(stream)));
   TCA_CHECK_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-  return word == 0 ? TCA_OK : TCA_ERR_TIMEOUT;
+  return word == 0 ? TCA_OK : (word == kStatusBounds ? TCA_ERR_BOUNDS : TCA_ERR_TIMEOUT);
 }
 
 }  // extern "C"

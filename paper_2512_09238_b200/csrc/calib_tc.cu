@@ -251,9 +251,7 @@ calib_rowstats_kernel(const CUtensorMap* __restrict__ maps, float* __restrict__ 
   ptx::tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    if (tid == 0) atomicExch(status, 1);
-    for (int k = 0; k < 64; ++k) __nanosleep(2000);  // let copies that are still in flight land
-    __syncthreads();
+    ptx::abort_teardown(status, tid);   // status word, then time for copies in flight to land
   }
   if (warp == 0) ptx::tmem_dealloc(tmem_base, 256);
 }
@@ -437,9 +435,7 @@ calib_colsum_kernel(const CUtensorMap* __restrict__ maps, const float* __restric
   ptx::tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    if (tid == 0) atomicExch(status, 1);
-    for (int i = 0; i < 64; ++i) __nanosleep(2000);  // let copies that are still in flight land
-    __syncthreads();
+    ptx::abort_teardown(status, tid);   // status word, then time for copies in flight to land
   } else {
     // every MMA has completed (each chain waited for its last S), so the K tile's shared memory
     // can carry chain 1's sums over to chain 0
@@ -456,8 +452,10 @@ calib_colsum_kernel(const CUtensorMap* __restrict__ maps, const float* __restric
 }
 
 
-// a[u] = sum of colmean[u] over the unit's selected indices / sum over its candidates [0, mb).
-// One CTA per unit; strided partial sums and a fixed-shape tree, hence reproducible.
+// a[u] of Eq. 4 as the share of the column means that the retained set holds: the unit's selected
+// indices plus its always-kept tail [mb, L), over all L tokens (Section 4.3 counts the global and
+// the local subset as retained).  One CTA per unit; strided partial sums and a fixed-shape tree,
+// hence reproducible.
 __global__ void __launch_bounds__(256)
 calib_score_kernel(const double* __restrict__ colmean, int64_t L, int64_t mb, const int32_t* __restrict__ idx,
                    const int64_t* __restrict__ offsets, double* __restrict__ a_out) {
@@ -466,7 +464,11 @@ calib_score_kernel(const double* __restrict__ colmean, int64_t L, int64_t mb, co
   const int64_t i0 = offsets[u], i1 = offsets[u + 1];
   double num = 0.0, den = 0.0;
   for (int64_t i = i0 + tid; i < i1; i += 256) num += c[idx[i]];
-  for (int64_t k = tid; k < mb; k += 256) den += c[k];
+  for (int64_t k = tid; k < L; k += 256) {
+    const double v = c[k];
+    den += v;
+    if (k >= mb) num += v;
+  }
   __shared__ double s_num[256], s_den[256];
   s_num[tid] = num;
   s_den[tid] = den;
@@ -504,7 +506,6 @@ int launch_colmean(const tca_params* prm, const void* Q, const void* K, int64_t 
   const CalibWs w = calib_ws_layout(prm, L, ws);
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int64_t heads = int64_t(prm->batch) * prm->n_q_heads;
-  TCA_CHECK_CUDA(cudaMemsetAsync(ws, 0, 256, stream));   // status word
   CUtensorMap maps[2];
   if (!encode_map(&maps[0], Q, D, L, heads, L) || !encode_map(&maps[1], K, D, L, U, L)) return TCA_ERR_CUDA;
   // pageable source: staged by the runtime before the call returns
@@ -556,7 +557,7 @@ extern "C" int tca_calib_score(const tca_params* prm, const double* colmean, int
                                const int64_t* offsets_dev, double* a_out, void* stream) {
   int st = check_params(prm);
   if (st != TCA_OK) return st;
-  TCA_CHECK_ARG(colmean && idx && offsets_dev && a_out && L >= 1);
+  TCA_CHECK_ARG(colmean && offsets_dev && a_out && L >= 1);   // idx may be NULL when nothing is selected
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int64_t mb = num_blocks(prm, L) * prm->block;
   calib_score_kernel<<<unsigned(U), 256, 0, static_cast<cudaStream_t>(stream)>>>(colmean, L, mb, idx, offsets_dev,

@@ -9,6 +9,8 @@
 
 namespace tca {
 
+constexpr int kStatusTimeout = 1;  // values of a workspace's status word
+constexpr int kStatusBounds = 2;
 constexpr int kMaxGroup = 8;    // query heads per KV head
 constexpr int kMaxBlock = 128;  // b
 
@@ -65,6 +67,7 @@ SelectWs select_ws_layout(const tca_params* prm, int64_t L, void* ws);
 // decode: a 256-byte header (word 0: sticky error flag, set when a bounded wait gave up)
 // followed by one partial (acc[d], max, sum) per (slice, query head of the group).
 constexpr int kDecodeChunkRows = 256;  // smallest slice of cache rows one CTA takes
+constexpr size_t kDecodeHeaderBytes = 256;
 struct DecodeWs {
   int* status;
   float* partial;     // [n_chunks_max][G][d + 2]

@@ -348,6 +348,23 @@ decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restri
   }
 }
 
+// Streaming multiprocessors of the current device, looked up once per device.
+constexpr int kMaxDevices = 64;
+std::mutex g_device_mutex;
+int g_sm_count[kMaxDevices] = {};
+
+inline int sm_count() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (g_sm_count[dev] == 0) {
+    int n = 0;
+    g_sm_count[dev] =
+        (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+  }
+  return g_sm_count[dev];
+}
+
 // Rows per CTA: enough CTAs for two per SM, at least one softmax round each.
 inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_sm, int64_t* max_len_out) {
   int64_t total = 0, max_len = 0;
@@ -357,15 +374,7 @@ inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_s
     max_len = len > max_len ? len : max_len;
   }
   *max_len_out = max_len;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      sms = n;
-    else
-      sms = 148;
-  }
+  const int sms = sm_count();
   // Smallest slice length for which the slices of all units fit the resident CTAs in one
   // wave: with one slice more than that, the extra CTA starts only after another one ends.
   const int64_t slots = int64_t(ctas_per_sm) * sms;
@@ -462,7 +471,6 @@ namespace tca {
 namespace {
 
 constexpr size_t kStaticScratchBytes = size_t(TCA_DECODE_STATIC_SCRATCH_BYTES);
-constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
 
@@ -516,4 +524,18 @@ extern "C" int tca_attn_decode_static(const tca_params* prm, const void* q, cons
   }
   if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, target, s);
   return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, target, s);
+}
+
+extern "C" int tca_decode_static_status(void* stream) {
+  void* scratch = nullptr;
+  int st = static_scratch(&scratch);
+  if (st != TCA_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t word = 0;
+  TCA_CHECK_CUDA(cudaMemcpyAsync(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost, s));
+  TCA_CHECK_CUDA(cudaStreamSynchronize(s));
+  if (word == 0) return TCA_OK;
+  TCA_CHECK_CUDA(cudaMemsetAsync(scratch, 0, sizeof(word), s));   // reported once: the word starts clean again
+  TCA_CHECK_CUDA(cudaStreamSynchronize(s));
+  return TCA_ERR_TIMEOUT;
 }

@@ -19,19 +19,18 @@ extern "C" int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const
                                      void* ws, size_t ws_bytes, void* stream) {
   int st = check_params(prm);
   if (st != TCA_OK) return st;
+  if (prm->window < 1) return TCA_ERR_UNSUPPORTED;  // a query always sees itself through its local subset
   TCA_CHECK_ARG(Q && K && V && c && O && ws);
   TCA_CHECK_ARG(c->k && c->v && c->pos && c->state);
   TCA_CHECK_ARG(L >= 1 && L < (int64_t(1) << 31));
   TCA_CHECK_ARG(row_begin >= 0 && row_begin < row_end && row_end <= L && row_begin % TCA_PREFILL_ROW_ALIGN == 0);
-  TCA_CHECK_ARG(prm->window >= 1);  // a query always sees itself through its local subset
   TCA_CHECK_ARG(aligned(Q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(O, 16) && aligned(ws, 256));
   TCA_CHECK_ARG(aligned(c->k, 16) && aligned(c->v, 16));
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   TCA_CHECK_ARG(c->n_units == U);
   TCA_CHECK_ARG(int64_t(prm->batch) * prm->n_q_heads <= 65535);
   if (ws_bytes < tca_workspace_bytes(prm, L, TCA_OP_PREFILL)) return TCA_ERR_WORKSPACE;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return TCA_ERR_CUDA;  // status word
+  cudaStream_t s = static_cast<cudaStream_t>(stream);   // word 0 of ws is the sticky status word: not cleared here
   if (prm->dtype == TCA_F32) {
     if (prm->head_dim == 128) return launch_prefill_simt<float, 128>(prm, Q, K, V, L, row_begin, row_end, c, O, s);
     return launch_prefill_simt<float, 64>(prm, Q, K, V, L, row_begin, row_end, c, O, s);

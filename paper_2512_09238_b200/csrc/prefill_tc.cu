@@ -367,9 +367,7 @@ prefill_tc_kernel(const CUtensorMap* __restrict__ maps, const int32_t* __restric
   ptx::tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    if (tid == 0) atomicExch(status, 1);
-    for (int i = 0; i < 64; ++i) __nanosleep(2000);  // let copies that are still in flight land
-    __syncthreads();
+    ptx::abort_teardown(status, tid);   // status word, then time for copies in flight to land
   }
   if (warp == 0) ptx::tmem_dealloc(tmem_base, 512);
 }

@@ -1,6 +1,7 @@
 // Thin inline-PTX wrappers for sm_100a: mbarrier, TMA tensor loads, tcgen05 (UMMA, TMEM).
-// Every wait is bounded: after kWaitLimitNs of polling it gives up and reports failure so
-// that the caller can raise a status flag, drain and exit instead of hanging the GPU.
+// Every wait is bounded: after its limit (kWaitLimitNs unless the caller passes another) it gives
+// up and reports failure so that the caller can raise a status flag, drain and exit instead of
+// hanging the GPU.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -46,19 +47,32 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait in these kernels
-// Returns false when the wait gave up (or *abort_flag was already set by another thread).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Returns false when the wait gave up after `limit_ns` (or *abort_flag was already set by another
+// thread); in the first case it also sets *abort_flag, so that every other waiter of the CTA
+// leaves its own wait at its next probe.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) break;
+      if (global_timer_ns() - t0 > limit_ns) break;
     }
   }
   *abort_flag = 1;
   return false;
+}
+
+// What a tensor-core kernel does once its CTA has met again after an aborted wait: raise the
+// status word the host reads, then give bulk copies that were already issued time to land before
+// the shared memory they target is handed back.  (TMEM is freed by the caller, as on the normal
+// path.)  Must be reached by every thread of the CTA.
+__device__ __forceinline__ void abort_teardown(int* status, int tid) {
+  if (tid == 0) atomicExch(status, 1);
+  for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  __syncthreads();
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {

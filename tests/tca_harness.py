@@ -98,7 +98,7 @@ def gpu_decode(run: DeviceRun, q: torch.Tensor) -> torch.Tensor:
     out = torch.empty_like(q)
     ws = B.alloc_workspace(run.prm, run.cache.rows_total, B.TCA_OP_DECODE)
     B.tca_attn_decode(run.prm, q, run.cache, out, ws)
-    torch.cuda.synchronize()
+    assert B.tca_ws_status(ws) == B.TCA_OK          # synchronises; a wait that gave up would leave stale partials
     return out
 
 

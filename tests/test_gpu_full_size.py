@@ -231,6 +231,16 @@ def test_calibration_column_means_at_32k():
                 want[:r + 1] += a[L - n_last:j + 1]
         want /= G * (n_last - np.arange(n_last))
         np.testing.assert_allclose(c[u, L - n_last:], want, rtol=2e-3, atol=1e-12)
+    # columns sampled over the whole range (first, around the window, tile edges, random, last) for
+    # one unit against the oracle: every visible row's softmax is normalised over all of its keys
+    rng = np.random.default_rng(5)
+    cols = sorted({0, 1, 2, 3, 127, 128, 129, wl.window - 1, wl.window, wl.window + 1, 16383, 16384, L - 129,
+                   L - 128, L - 2, L - 1} | {int(x) for x in rng.integers(0, L, size=64)})
+    u = 3
+    s_, h_ = divmod(u, wl.n_kv_heads)
+    want = O.attention_column_means_at(I.widen(data["q"][s_, h_ * G:(h_ + 1) * G, :L]), I.widen(data["k"][s_, h_, :L]),
+                                       scale, cols, rows_per_step=1024)
+    np.testing.assert_allclose(c[u, cols], want, rtol=2e-3, atol=1e-12)
     # Eq. 4 for two budgets through the library's own selection
     B.tca_score(pipe.prm, pipe.q_last, pipe.Kp, L, pipe.logscore, pipe.ws_score)
     a_prev = None
@@ -250,3 +260,35 @@ def test_calibration_column_means_at_32k():
             np.testing.assert_allclose(a, 1.0, rtol=1e-12)
             assert np.all(a >= a_prev)
         a_prev = a
+
+
+def test_calibration_column_means_at_128k():
+    """The same dense passes at the benchmark length, L = 131072 (config 4): row sums, and the last 96
+    columns (seen fully by the last 96 rows) against the definition for both end units."""
+    wl = I.WORKLOADS["config4"].scaled(decode_steps=0)
+    data, p, pipe = _pipeline(wl)
+    L, U, G = wl.L, pipe.U, wl.group
+    col = torch.empty(U, L, dtype=torch.float64, device="cuda")
+    ws = B.alloc_workspace(pipe.prm, L, B.TCA_OP_CALIB)
+    B.tca_calib_colmean(pipe.prm, pipe.Qp, pipe.Kp, L, col, ws)
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(ws) == B.TCA_OK
+    c = col.cpu().numpy()
+    assert np.all(np.isfinite(c)) and np.all(c >= 0)
+    np.testing.assert_allclose((c * (L - np.arange(L))).sum(1), float(L), rtol=1e-5)
+    scale = H.scale_of(wl)
+    n_last = 96
+    for u in (0, U - 1):
+        s, h = divmod(u, wl.n_kv_heads)
+        K = I.widen(data["k"][s, h, :L])
+        want = np.zeros(n_last)
+        for g in range(G):
+            Q = I.widen(data["q"][s, h * G + g, L - n_last:L])
+            for r in range(n_last):
+                j = L - n_last + r
+                x = (K[:j + 1] @ Q[r]) * scale
+                a = np.exp(x - x.max())
+                a /= a.sum()
+                want[:r + 1] += a[L - n_last:j + 1]
+        want /= G * (n_last - np.arange(n_last))
+        np.testing.assert_allclose(c[u, L - n_last:], want, rtol=2e-3, atol=1e-12)

@@ -104,6 +104,14 @@ def test_compaction_is_bit_exact(runs, name):
 
 
 def _oracle_T(run, wl, u):
+    """The retained set the oracle's attention is evaluated on: the index set the GPU selected.
+
+    Selection has its own tests (test_selection_matches_oracle compares the GPU's index set with
+    the oracle's under the 1e-5 rule: equal, or different only where the oracle's scores at the
+    budget boundary are closer than 1e-5).  The attention tests then ask a separate question: given
+    an index set, is the attention over it right?  Feeding both sides the GPU's set keeps an
+    accepted boundary difference in the selection from showing up a second time as an attention
+    error, and hides nothing, because a wrong set already fails the selection test."""
     idx = run.idx.cpu().numpy()
     S = idx[run.offsets[u]:run.offsets[u + 1]].astype(np.int64)
     return O.retained_set(S, run.m, wl.block, wl.L)
@@ -236,6 +244,76 @@ def test_degenerate_lengths(L, w, b):
         want = O.attention_rows(I.widen(data["q"][0, h]), I.widen(data["k"][0, h]), I.widen(data["v"][0, h]),
                                 res["T"], w, H.scale_of(wl))
         H.check_attention(out[0, h], want, "f32", f"L={L}")
+
+
+@pytest.mark.parametrize("d,G", [(64, 2), (128, 4)])
+@pytest.mark.parametrize("L,w,b", [(100, 128, 32),    # w >= L: no blocks at all, n_global = 0
+                                   (1, 4, 4),         # a single token
+                                   (100, 16, 32),     # L below one 128-row tile, two blocks
+                                   (129, 1, 128),     # one row into the second tile, w = 1, one block of 128
+                                   (300, 40, 64),     # a global region shorter than one key tile
+                                   (257, 300, 16)])   # w >= L across three query tiles
+def test_degenerate_lengths_on_the_tensor_core_paths(L, w, b, d, G):
+    """bf16 inputs, so the prefill runs on the tcgen05 kernel and the decode on the mma.sync kernel:
+    every output row against the oracle on the method's edge cases."""
+    wl = BASE.scaled(batch=1, n_q_heads=2 * G, n_kv_heads=2, head_dim=d, L=L, window=w, block=b, dtype="bf16",
+                     seed=32, budget=("fixed", 0.5))
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    run = H.gpu_select_compact(wl, data, p)
+    out = H.from_device(H.gpu_prefill(run))
+    dec = H.from_device(H.gpu_decode(run, run.dev["q"][:, :, L - 1, :].contiguous()))
+    scale = H.scale_of(wl)
+    for h in range(2):
+        res = H.oracle_select_unit(wl, data, p, 0, h, L)
+        assert res["m"] == max(0, (L - w) // b)
+        S = run.idx.cpu().numpy()[run.offsets[h]:run.offsets[h + 1]].astype(np.int64)
+        assert H.compare_selection(res, S, run.t.cpu().numpy()[h, :res["m"]], b) == 0
+        K, V = I.widen(data["k"][0, h]), I.widen(data["v"][0, h])
+        for g in range(G):
+            Q = I.widen(data["q"][0, h * G + g])
+            want = O.attention_rows(Q, K, V, res["T"], w, scale)
+            H.check_attention(out[0, h * G + g], want, "bf16", f"prefill L={L} w={w} b={b} d={d}")
+            want_dec = O.attention_over_set(Q[L - 1], K[res["T"]], V[res["T"]], scale)
+            H.check_attention(dec[0, h * G + g], want_dec, "bf16", f"decode L={L} w={w} b={b} d={d}")
+
+
+def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_gpu_usable():
+    """Every mbarrier wait of the tensor-core kernels has a time limit and one way out.  The
+    self-test entry point runs that way out in miniature (a wait of about a millisecond on a
+    barrier nothing arrives at): the call must return, the status word must read TCA_ERR_TIMEOUT,
+    and a prefill and a decode afterwards must still be right."""
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    assert B.tca_ws_status(ws) == B.TCA_OK
+    B.tca_selftest_wait_expiry(ws, 1_000_000, waited)
+    assert B.tca_ws_status(ws) == B.TCA_ERR_TIMEOUT                  # synchronises: the kernel has returned
+    assert 1_000_000 <= int(waited.item()) < 1_000_000_000           # gave up after the limit, well inside a second
+    assert B.tca_ws_status(ws) == B.TCA_ERR_TIMEOUT                  # sticky until the caller clears it
+    with pytest.raises(B.TcaError):
+        B.tca_selftest_wait_expiry(ws, 10, waited)                   # limits outside 1 us .. 100 ms are refused
+    # a prefill on a workspace whose status word is set returns at once and leaves O alone
+    wl = SMALL["bf16_d64_g2"]
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    run = H.gpu_select_compact(wl, data, p)
+    ws_bad = B.alloc_workspace(run.prm, run.L, B.TCA_OP_PREFILL)
+    ws_bad[:4] = torch.tensor([1, 0, 0, 0], dtype=torch.uint8, device="cuda")
+    O_dev = torch.full_like(run.dev["q"], 7.0)
+    B.tca_attn_prefill(run.prm, run.dev["q"], run.dev["k"], run.dev["v"], run.L, run.cache, O_dev, ws_bad)
+    assert B.tca_ws_status(ws_bad) == B.TCA_ERR_TIMEOUT
+    assert bool((O_dev == 7.0).all())
+    # and the device is fine: the normal paths still match the oracle
+    out = H.from_device(H.gpu_prefill(run))
+    dec = H.from_device(H.gpu_decode(run, run.dev["q"][:, :, wl.L - 1, :].contiguous()))
+    scale, G = H.scale_of(wl), wl.group
+    for h in range(wl.n_kv_heads):
+        T = _oracle_T(run, wl, h)
+        K, V = I.widen(data["k"][0, h, :wl.L]), I.widen(data["v"][0, h, :wl.L])
+        Q = I.widen(data["q"][0, h * G, :wl.L])
+        H.check_attention(out[0, h * G], O.attention_rows(Q, K, V, T, wl.window, scale), "bf16", "prefill after expiry")
+        H.check_attention(dec[0, h * G], O.attention_over_set(Q[wl.L - 1], K[T], V[T], scale), "bf16",
+                          "decode after expiry")
 
 
 @pytest.mark.parametrize("name,steps", [("bf16_gqa4", 150), ("bf16_d64_g2", 40), ("f32_g3_b1", 20),

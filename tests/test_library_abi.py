@@ -86,6 +86,30 @@ def test_parameter_validation_happens_on_the_host():
     assert L.tca_score(ctypes.byref(bad), None, None, 2048, None, None, 0, None) == B.TCA_ERR_UNSUPPORTED
 
 
+def test_prefill_refuses_a_zero_window_before_touching_anything():
+    """With w = 0 a query that is not selected itself would attend to nothing; the prefill entry
+    points say so (the other calls accept w = 0).  The check precedes every pointer check."""
+    w0 = B.make_params(1, 8, 8, 64, 32, 0)
+    L = B.lib()
+    assert L.tca_attn_prefill(ctypes.byref(w0), None, None, None, 2048, None, None, None, 0, None) == B.TCA_ERR_UNSUPPORTED
+    assert L.tca_attn_prefill_rows(ctypes.byref(w0), None, None, None, 2048, 0, 128, None, None, None, 0,
+                                   None) == B.TCA_ERR_UNSUPPORTED
+    assert B.tca_workspace_bytes(w0, 2048, B.TCA_OP_SELECT) > 0
+    w1 = B.make_params(1, 8, 8, 64, 32, 1)
+    assert L.tca_attn_prefill(ctypes.byref(w1), None, None, None, 2048, None, None, None, 0, None) == B.TCA_ERR_INVALID_ARG
+
+
+def test_static_decode_limit_formula_is_the_workspace_size():
+    """The limit documented for tca_attn_decode_static is tca_workspace_bytes for TCA_OP_DECODE."""
+    def up(x):
+        return (x + 255) // 256 * 256
+    for (batch, hq, hkv, d, rows) in [(1, 32, 8, 128, 500000), (2, 8, 2, 64, 12345), (4, 7, 1, 128, 256)]:
+        prm = B.make_params(batch, hq, hkv, d, 64, 512)
+        U, G = batch * hkv, hq // hkv
+        want = 256 + up((rows // 256 + 2 * U + 1) * G * (d + 2) * 4)
+        assert B.tca_workspace_bytes(prm, rows, B.TCA_OP_DECODE) == want
+
+
 def test_workspace_sizes_scale_as_documented():
     prm = B.make_params(1, 32, 8, 128, 128, 4096)
     L = 131072

@@ -403,6 +403,19 @@ def test_column_means_against_a_masked_dense_matrix():
     assert float(np.sum(c1 * (L - np.arange(L)))) == pytest.approx(L, rel=1e-12)
 
 
+def test_sampled_column_means_equal_the_full_evaluation():
+    """The chunked, sampled-column form used at long sequence lengths is the same function: equal
+    to the row-by-row evaluation on every column, for chunk sizes that do and do not divide L."""
+    rng = _rng(24)
+    L, d, G = 61, 6, 2
+    Q, K = rng.standard_normal((G, L, d)) * 1.3, rng.standard_normal((L, d)) * 1.3
+    full = O.attention_column_means(Q, K, 0.45)
+    for step in (1, 7, 16, 61, 100):
+        np.testing.assert_allclose(O.attention_column_means_at(Q, K, 0.45, np.arange(L), step), full, rtol=1e-12)
+    cols = np.array([0, 5, 17, 59, 60])
+    np.testing.assert_allclose(O.attention_column_means_at(Q, K, 0.45, cols, 8), full[cols], rtol=1e-12)
+
+
 def test_aggregated_score_is_the_retained_share_of_all_column_means():
     """4 candidates and 2 always-kept tail tokens, values chosen so that the plain sum of Eq. 4
     (0.625), a share of the candidates only (0.625 / 1.125), a share of everything without the

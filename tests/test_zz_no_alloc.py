@@ -48,6 +48,9 @@ def test_static_decode_matches_workspace_decode_twice_in_a_row():
     B.tca_attn_decode_static(run.prm, q1, run.cache, again)
     torch.cuda.synchronize()
     assert torch.equal(again, got1)
+    # no bounded wait gave up in any of the three calls (the only place this variant can say so)
+    assert B.tca_decode_static_status() == B.TCA_OK
+    assert torch.cuda.mem_get_info()[0] >= free_before
 
 
 def test_static_decode_refuses_caches_beyond_its_scratch():
