@@ -58,7 +58,8 @@ __all__ = [
     "select_tokens", "retained_set", "select_head", "visible_mask_row",
     "attention_rows", "attention_over_set", "candidate_grid", "DecodeCache",
     "dropped_mass", "attention_column_means", "attention_column_means_at", "aggregated_score",
-    "calibrate_head",
+    "calibrate_head", "block_metric_entropy", "random_block_keys", "select_tokens_flat",
+    "select_head_variant",
 ]
 
 
@@ -417,3 +418,77 @@ class DecodeCache:
         """One decode step for one query head: attention over the whole retained cache."""
         pos = self.positions()
         return attention_over_set(q, K_all[pos], V_all[pos], self.sm_scale)
+
+
+# ----------------------------------------------------------------------------- ablation variants
+# The appendix ("Effectiveness of Local-context Redundancy Metric", "Ablations on Concentration
+# Index") compares the method with two variants it does not spell out: a block-wise entropy in
+# place of the Herfindahl-Hirschman term of Eq. 6, and blocks "randomly sorted" instead of sorted
+# by h.  A third variant, one flat top-B over all candidates of a head, is what "a per-head
+# budgeted top-k" means when read without the block structure.  Readings (parity unpinned against
+# the authors' code, which the paper does not show): entropy = Shannon entropy (natural log) of the
+# block's scores normalised inside the block, unscaled; random order = blocks ranked by a seeded
+# 64-bit hash of (seed, head unit, block index); flat = the B best candidates, ties to the lower
+# index, with B the size of the global subset the configuration gives.
+def block_metric_entropy(log_s: np.ndarray, m: int, b: int, alpha: float) -> np.ndarray:
+    """Eq. 6 with the block entropy as concentration index:
+    h_j = (1 - alpha) * sum_i s_i + alpha * H_j,  H_j = -sum_i p_i ln p_i,  p_i = s_i / sum_{B_j} s."""
+    h = np.empty(m, dtype=np.float64)
+    for j in range(m):
+        l = np.asarray(log_s[j * b:(j + 1) * b], dtype=np.float64)
+        top = float(np.max(l))
+        e = np.exp(l - top)
+        mass = math.exp(top) * float(np.sum(e))
+        pr = e / np.sum(e)
+        nz = pr > 0.0                                    # 0 * ln 0 = 0
+        entropy = -float(np.sum(pr[nz] * np.log(pr[nz])))
+        h[j] = (1.0 - alpha) * mass + alpha * entropy
+    return h
+
+
+def _splitmix64(x: int) -> int:
+    """The SplitMix64 finaliser (Steele, Lea, Flood 2014), a published 64-bit mixing function."""
+    mask = (1 << 64) - 1
+    x = (x + 0x9E3779B97F4A7C15) & mask
+    x = ((x ^ (x >> 30)) * 0xBF58476D1CE4E5B9) & mask
+    x = ((x ^ (x >> 27)) * 0x94D049BB133111EB) & mask
+    return x ^ (x >> 31)
+
+
+def random_block_keys(seed: int, unit: int, m: int) -> np.ndarray:
+    """Sort keys of the random-order variant: for block j of head unit `unit`,
+    key = SplitMix64(SplitMix64(seed * 2^32 + unit) + j) >> 11, scaled to [0, 1).  Blocks are
+    then ranked ascending by (key, j) exactly as they are by (h, j) in the method proper."""
+    base = _splitmix64(((int(seed) & 0xFFFFFFFF) << 32) | (int(unit) & 0xFFFFFFFF))
+    mask = (1 << 64) - 1
+    return np.array([(_splitmix64((base + j) & mask) >> 11) * 2.0 ** -53 for j in range(m)], dtype=np.float64)
+
+
+def select_tokens_flat(log_s: np.ndarray, n_keep: int, n_candidates: int) -> np.ndarray:
+    """The n_keep highest-scoring tokens among the candidates [0, n_candidates), ties to the lower
+    index, ascending: the whole candidate range treated as one block of Eq. 8."""
+    cand = np.asarray(log_s[:n_candidates], dtype=np.float64)
+    order = np.argsort(-cand, kind="stable")[:int(n_keep)]
+    return np.sort(order).astype(np.int64)
+
+
+def select_head_variant(q_last, K, p, b: int, w: int, alpha: float, sm_scale: float, variant: str,
+                        seed: int = 0, unit: int = 0):
+    """select_head for one of the variants: "entropy", "random" or "flat"."""
+    L = K.shape[0]
+    m = num_blocks(L, b, w)
+    log_s = log_importance(q_last, K, sm_scale)
+    n = resolve_counts(p, m)
+    if variant == "flat":
+        n_keep = int(np.sum(retain_counts(b) * n))
+        S = select_tokens_flat(log_s, n_keep, m * b)
+        return {"log_s": log_s, "m": m, "n": n, "S": S, "T": retained_set(S, m, b, L)}
+    if variant == "entropy":
+        h = block_metric_entropy(log_s, m, b, alpha)
+    elif variant == "random":
+        h = random_block_keys(seed, unit, m)
+    else:
+        raise ValueError(f"unknown variant {variant!r}")
+    t = block_requirement(h, n, b)
+    S = select_tokens(log_s, t, b)
+    return {"log_s": log_s, "m": m, "h": h, "n": n, "t": t, "S": S, "T": retained_set(S, m, b, L)}

@@ -468,3 +468,86 @@ def test_calibration_picks_the_sparsest_candidate_that_reaches_tau():
     # a threshold nothing reaches falls back to the last candidate; equal sizes go to the lower index
     assert O.calibrate_head(Q, K, cands[:2], b, w, 0.5, 0.99999, 1.0)[0] == 1
     assert O.calibrate_head(Q, K, np.stack([cands[1], cands[1]]), b, w, 0.5, 0.5, 1.0)[0] == 0
+
+
+# ----------------------------------------------------------------------------- ablation variants
+@pytest.mark.parametrize("b", [4, 32, 128])
+def test_entropy_index_closed_forms(b):
+    """Uniform block: H = ln b; one-hot block: H = 0; two equal scores: ln 2; a common factor on
+    the block's scores leaves H unchanged; with alpha = 1 the metric is H alone."""
+    uniform = np.full(b, math.log(1.0 / (3 * b)))
+    onehot = np.full(b, -700.0)
+    onehot[b // 2] = math.log(0.2)
+    two = np.full(b, -700.0)
+    two[0] = two[b - 1] = math.log(0.1)
+    ls = np.concatenate([uniform, onehot, two, uniform + 2.5])
+    h = O.block_metric_entropy(ls, 4, b, 1.0)
+    assert h[0] == pytest.approx(math.log(b), rel=1e-12)
+    assert h[1] == pytest.approx(0.0, abs=1e-12)
+    assert h[2] == pytest.approx(math.log(2.0), rel=1e-12)
+    assert h[3] == pytest.approx(h[0], rel=1e-12)                    # scale invariance
+    mass = O.block_metric_entropy(ls, 4, b, 0.0)                     # alpha = 0: the mass term, as in Eq. 6
+    np.testing.assert_allclose(mass, O.block_metric(ls, 4, b, 0.0), rtol=1e-14)
+    assert mass[0] == pytest.approx(1.0 / 3.0, rel=1e-12)
+    # against SciPy's entropy of the normalised block
+    rng = _rng(31)
+    x = rng.standard_normal(3 * b) * 2
+    from scipy.stats import entropy as sp_entropy
+    want = [sp_entropy(sp_softmax(x[j * b:(j + 1) * b])) for j in range(3)]
+    np.testing.assert_allclose(O.block_metric_entropy(x, 3, b, 1.0), want, rtol=1e-12)
+
+
+def test_random_order_is_a_seeded_permutation_of_psi():
+    """The random-order variant hands out exactly the counts of Psi (a permutation of it), the
+    same ones for the same seed, different ones for another seed or another head unit."""
+    m, b = 40, 8
+    n = O.resolve_counts([0.4, 0.3, 0.2, 0.1], m)
+    psi = O.budget_map(n, b)
+    k0 = O.random_block_keys(7, 3, m)
+    assert np.all((k0 >= 0) & (k0 < 1)) and len(np.unique(k0)) == m
+    t0 = O.block_requirement(k0, n, b)
+    np.testing.assert_array_equal(np.sort(t0), psi)
+    np.testing.assert_array_equal(O.block_requirement(O.random_block_keys(7, 3, m), n, b), t0)
+    assert not np.array_equal(O.block_requirement(O.random_block_keys(8, 3, m), n, b), t0)
+    assert not np.array_equal(O.block_requirement(O.random_block_keys(7, 4, m), n, b), t0)
+    # the mixing function against its published test vector: SplitMix64 seeded with 0 gives
+    # 0xE220A8397B1DCDAF as its first output
+    assert O._splitmix64(0) == 0xE220A8397B1DCDAF
+    # keys do not depend on the scores: the order is independent of h
+    rng = _rng(32)
+    h = rng.random(m)
+    assert not np.array_equal(O.rank_blocks(h), O.rank_blocks(k0))
+
+
+def test_flat_top_b_is_a_truncated_stable_argsort_and_a_best_subset():
+    rng = _rng(33)
+    ls = np.round(rng.standard_normal(24), 1)                 # rounded: ties exist
+    S = O.select_tokens_flat(ls, 7, 20)
+    assert np.all(np.diff(S) > 0) and len(S) == 7 and S.max() < 20
+    np.testing.assert_array_equal(S, np.sort(np.lexsort((np.arange(20), -ls[:20]))[:7]))
+    # best subset by brute force on a tiny tie-free case
+    import itertools
+    x = rng.standard_normal(9)
+    best = max(itertools.combinations(range(8), 3), key=lambda c: sum(x[list(c)]))
+    np.testing.assert_array_equal(O.select_tokens_flat(x, 3, 8), np.array(best))
+    # ties go to the lower index; nothing outside the candidates is ever taken
+    tie = np.array([1.0, 5.0, 5.0, 5.0, 0.0, 9.0])
+    np.testing.assert_array_equal(O.select_tokens_flat(tie, 2, 5), [1, 2])
+    # one block covering all candidates: the block-wise rule gives the same set
+    np.testing.assert_array_equal(O.select_tokens_flat(x, 3, 8), O.select_tokens(x, [3], 8))
+
+
+def test_variant_heads_keep_the_budget_and_differ_from_the_method():
+    rng = _rng(34)
+    L, d, G, b, w = 200, 16, 2, 8, 24
+    K = rng.standard_normal((L, d)) * 1.5
+    q = rng.standard_normal((G, d)) * 1.5
+    p = np.array([0.4, 0.3, 0.2, 0.1])
+    base = O.select_head(q, K, p, b, w, 0.5, 0.25)
+    for variant in ("entropy", "random", "flat"):
+        r = O.select_head_variant(q, K, p, b, w, 0.5, 0.25, variant, seed=5, unit=1)
+        assert len(r["S"]) == len(base["S"]) and np.all(np.diff(r["S"]) > 0) and r["S"].max() < base["m"] * b
+        assert not np.array_equal(r["S"], base["S"])
+    flat = O.select_head_variant(q, K, p, b, w, 0.5, 0.25, "flat")
+    dropped = np.setdiff1d(np.arange(base["m"] * b), flat["S"])
+    assert base["log_s"][flat["S"]].min() >= base["log_s"][dropped].max()
