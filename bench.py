@@ -149,6 +149,7 @@ class Pipeline:
         self.idx = torch.empty(max(1, int(self.offsets[-1])), dtype=torch.int32, device="cuda")
         self.ws_score = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_SCORE)
         self.ws_select = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_SELECT)
+        self.ws_score_select = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_SCORE_SELECT)
         self.ws_prefill = B.alloc_workspace(self.prm, wl.L, B.TCA_OP_PREFILL)
         self.ws_decode = B.alloc_workspace(self.prm, self.cache.rows_total, B.TCA_OP_DECODE)
         # device views used by the step (Q/K/V of the prompt are the first L tokens)
@@ -180,7 +181,7 @@ class Pipeline:
             self.row_ranges = list(zip(cuts[:-1], cuts[1:]))[::-1]
             self.ws_rows = [B.alloc_workspace(self.prm, wl.L, B.TCA_OP_PREFILL) for _ in self.row_ranges]
             self.h_Od = torch.empty_like(self.h_qd).pin_memory()
-        self.launches_per_step = 2 + 3 + 1 + 1 + wl.decode_steps * 3   # score 2, select 3, compact, prefill; append + split + combine per step
+        self.launches_per_step = 4 + 1 + 1 + wl.decode_steps * 3   # score + select fused: 4, compact, prefill; append + split + combine per step
         self.ev = {}
 
     def _ev(self, name):
@@ -194,10 +195,9 @@ class Pipeline:
         B, prm, L = self.B, self.prm, self.L
         if mark: self._ev("t_begin")
         if mark: self._ev("t0")
-        B.tca_score(prm, self.q_last, self.Kp, L, self.logscore, self.ws_score)
-        if mark: self._ev("t_score")
-        B.tca_select(prm, self.logscore, L, self.n_k, self.idx, self.offsets_dev, None, None, self.ws_select)
-        if mark: self._ev("t_select")
+        B.tca_score_select(prm, self.q_last, self.Kp, L, self.n_k, self.logscore, self.idx, self.offsets_dev, None, None,
+                           self.ws_score_select)
+        if mark: self._ev("t_score_select")
         B.tca_compact_kv(prm, self.Kp, self.Vp, L, self.idx, self.offsets_dev, self.offsets, self.cache)
         if mark: self._ev("t_compact")
         B.tca_attn_prefill(prm, self.Qp, self.Kp, self.Vp, L, self.cache, self.O, self.ws_prefill)
@@ -242,10 +242,9 @@ class Pipeline:
             ev_dec = torch.cuda.Event(); ev_dec.record(self.s_in)
         cs.wait_event(ev_k)
         if mark: self._ev("t0")
-        B.tca_score(prm, self.q_last, self.Kp, L, self.logscore, self.ws_score)
-        if mark: self._ev("t_score")
-        B.tca_select(prm, self.logscore, L, self.n_k, self.idx, self.offsets_dev, None, None, self.ws_select)
-        if mark: self._ev("t_select")
+        B.tca_score_select(prm, self.q_last, self.Kp, L, self.n_k, self.logscore, self.idx, self.offsets_dev, None, None,
+                           self.ws_score_select)
+        if mark: self._ev("t_score_select")
         cs.wait_event(ev_v)
         B.tca_compact_kv(prm, self.Kp, self.Vp, L, self.idx, self.offsets_dev, self.offsets, self.cache)
         if mark: self._ev("t_compact")
@@ -273,7 +272,7 @@ class Pipeline:
 
     def stage_ms(self):
         """Mean milliseconds per stage over the marked steps."""
-        names = ["t_begin", "t0", "t_score", "t_select", "t_compact", "t_prefill", "t_prefill_io", "t_decode"]
+        names = ["t_begin", "t0", "t_score_select", "t_compact", "t_prefill", "t_prefill_io", "t_decode"]
         out = {}
         for a, b in zip(names[:-1], names[1:]):
             out["h2d" if b == "t0" else b[2:]] = float(np.mean([x.elapsed_time(y) for x, y in zip(self.ev[a], self.ev[b])]))
@@ -345,8 +344,15 @@ def calibration_leg(pipe, torch, B, sm_max_mhz, n_candidates: int = 14, tau: flo
     ex2_per_s = 2 * pairs / (colmean_ms * 1e-3)                     # both passes exponentiate every pair
     peak = 16 * 148 * sm_max_mhz * 1e6
     rows_sum = float((col[0] * (L - torch.arange(L, device="cuda", dtype=torch.float64))).sum().item())
+    # The same scores against lower thresholds: on these inputs the retained share of the score
+    # follows the retained share of the tokens, so tau = 0.9 is out of reach of the sparsest-to-densest
+    # sweep of Eq. 3 with sigma = 1 (its last candidate keeps 76 % of the candidates) and Algorithm 1 ends
+    # at its fall-back; lower thresholds take the valid branch.
+    sweep = {f"{t:.2f}": [B.tca_calib_choose(a[:, u], sizes[:, u], t) for u in range(U)] for t in (0.9, 0.8, 0.7, 0.5)}
     return {"colmean_ms": colmean_ms, "candidates_ms": e1.elapsed_time(e2), "n_candidates": n_candidates, "tau": tau,
-            "choice_per_unit": choice,
+            "choice_per_unit": choice, "choice_per_unit_by_tau": sweep,
+            "a_by_candidate_mean_over_units": [float(x) for x in a.mean(axis=1)],
+            "share_of_candidates_kept_by_candidate": [float(sizes[i, 0]) / (pipe.m * wl.block) for i in range(n_candidates)],
             "retained_share_of_candidates": [float(sizes[choice[u], u]) / (pipe.m * wl.block) for u in range(U)],
             "a_of_choice": [float(a[choice[u], u]) for u in range(U)],
             "row_sum_check_unit0": rows_sum / L,
@@ -500,7 +506,7 @@ def main():
     assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
     assert B.tca_ws_status(pipe.ws_decode) == B.TCA_OK     # no decode step timed on stale partials
     work = pipe.algorithmic_work()
-    prefill_ms = stages["score"] + stages["select"] + stages["compact"] + stages["prefill"]
+    prefill_ms = stages["score_select"] + stages["compact"] + stages["prefill"]
     value = job_throughput(world, wl.batch, wl.L, prefill_ms)
     decode_us = stages["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None   # no decode phase: no figure
 
@@ -526,8 +532,8 @@ def main():
         return {"ms": ms, "bytes": bytes_, "achieved_gbs": gbs, "frac_of_measured": gbs / hbm, "frac_of_8tbs": gbs / 8000.0}
 
     out["stages"] = {
-        "score": hbm_stage(work["score_bytes"], stages["score"]),
-        "select": {"ms": stages["select"]},
+        "score_select": dict(hbm_stage(work["score_bytes"], stages["score_select"]), launches=4,
+                             note="tca_score_select: logits, finalize + block metric, rank, top-t; bytes are the score's"),
         "compact": hbm_stage(work["compact_bytes"], stages["compact"]),
         "prefill": {"ms": stages["prefill"], "flops": work["prefill_flops"], "dense_flops": work["dense_prefill_flops"]},
         "decode_step": hbm_stage(work["decode_bytes_per_step"], decode_us * 1e-3) if decode_us else None,
@@ -541,7 +547,7 @@ def main():
         main_pipe = pipe
         pipe = Pipeline(dense_wl, data, I.budget_table(dense_wl), torch, B, host_io=False)
         _, st_dense, _ = timed(host_io=False)
-        dense_prefill = st_dense["score"] + st_dense["select"] + st_dense["compact"] + st_dense["prefill"]
+        dense_prefill = st_dense["score_select"] + st_dense["compact"] + st_dense["prefill"]
         dense_decode_us = st_dense["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None
         out["dense_baseline"] = {"budget": 1.0, "prefill_ms": dense_prefill, "decode_us_per_step": dense_decode_us,
                                  "speedup_prefill": dense_prefill / prefill_ms,
@@ -559,7 +565,7 @@ def main():
         nKV = wl.batch * wl.n_kv_heads * wl.head_dim * elt
         h2d = wl.L * (nQ + 2 * nKV) + nQ + wl.decode_steps * (nQ + 2 * nKV)   # prompt, newest query again, decode tokens
         d2h = wl.L * nQ + wl.decode_steps * nQ
-        e2e_prefill_ms = sum(st_e2e[k] for k in ("h2d", "score", "select", "compact", "prefill", "prefill_io"))
+        e2e_prefill_ms = sum(st_e2e[k] for k in ("h2d", "score_select", "compact", "prefill", "prefill_io"))
         out["e2e"] = {"value": job_throughput(world, wl.batch, wl.L, e2e_prefill_ms), "unit": UNIT,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                       "prefill_ms": e2e_prefill_ms,

@@ -54,13 +54,31 @@ enum {
 
 enum { TCA_F32 = 0, TCA_BF16 = 1 };
 
-/* tca_params.flags: run the prefill on the FP32 pipes even for bf16 inputs (the slow
- * reference kernel the tensor-core kernel is cross-checked against). */
-enum { TCA_FLAG_PREFILL_SIMT = 1 };
+/* tca_params.flags */
+enum {
+  /* run the prefill on the FP32 pipes even for bf16 inputs (the slow reference kernel the
+   * tensor-core kernel is cross-checked against) */
+  TCA_FLAG_PREFILL_SIMT = 1,
+  /* Selection variants of the paper's ablations (appendix "Ablations on Concentration Index" and
+   * "Effectiveness of Local-context Redundancy Metric") and a flat top-B; at most one of the three.
+   * The paper names them without formulas; the definitions here are this library's reading.
+   *   ENTROPY_INDEX  the concentration term of Eq. 6 becomes the block entropy
+   *                  H_j = -sum_i p_i ln p_i, p_i = s_i / sum_{B_j} s  (in place of 1 - sum p_i^2)
+   *   RANDOM_ORDER   blocks are ranked by a hash of (tca_params.seed, unit, block index) instead of
+   *                  h_j: key = SplitMix64(SplitMix64(seed * 2^32 + unit) + j) >> 11, ascending,
+   *                  ties to the lower block; h_out receives key * 2^-53
+   *   FLAT_TOPB      no blocks: the n_sel = sum_k k * n_k highest-scoring tokens among the candidates
+   *                  [0, m*b) are selected, ties to the lower position; h_out and t_out are not written */
+  TCA_FLAG_ENTROPY_INDEX = 2,
+  TCA_FLAG_RANDOM_ORDER = 4,
+  TCA_FLAG_FLAT_TOPB = 8,
+  /* prefill: walk each query tile's own window band before the selected keys (see tca_attn_prefill) */
+  TCA_FLAG_PREFILL_BAND_FIRST = 16
+};
 
 enum {
   TCA_OP_SCORE = 0, TCA_OP_SELECT = 1, TCA_OP_COMPACT = 2,
-  TCA_OP_PREFILL = 3, TCA_OP_DECODE = 4, TCA_OP_APPEND = 5, TCA_OP_CALIB = 6
+  TCA_OP_PREFILL = 3, TCA_OP_DECODE = 4, TCA_OP_APPEND = 5, TCA_OP_CALIB = 6, TCA_OP_SCORE_SELECT = 7
 };
 
 /* Hyper-parameters of one attention layer (Algorithm 2, REQUIRE line). */
@@ -75,6 +93,7 @@ typedef struct tca_params {
   float sm_scale;     /* 1/sqrt(d_h) of Eqs. 2 and 5                                    */
   int32_t dtype;      /* TCA_F32 or TCA_BF16: element type of Q, K, V, O and the cache  */
   int32_t flags;      /* 0, or TCA_FLAG_* bits                                          */
+  int32_t seed;       /* TCA_FLAG_RANDOM_ORDER: seed of the block order; otherwise unused    */
 } tca_params;
 
 /* Number of int64 words per unit in tca_cache_desc.state. */
@@ -123,6 +142,10 @@ typedef struct tca_cache_desc {
 const char* tca_strerror(int status);
 int tca_version(void);
 
+/* Bit flags describing how the library was built. */
+enum { TCA_BUILD_DEBUG_BOUNDS = 1 };
+int tca_build_info(void);
+
 /*
  * Budget map of Eq. 7 (Section 4.2), resolved on the host.
  *   p       HOST [n_kv_heads, nK] double: configuration over K = {1, 2, 4, ..., 2^(nK-1)};
@@ -170,6 +193,18 @@ int tca_score(const tca_params* prm, const void* q_last, const void* K, int64_t 
 int tca_select(const tca_params* prm, const double* logscore, int64_t L,
                const int32_t* n_k, int32_t nK, int32_t* idx, const int64_t* offsets_dev,
                double* h_out, int32_t* t_out, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * tca_score followed by tca_select in one call and fewer launches (Eqs. 5-8, Algorithm 2 lines
+ * 1-6): the kernel that turns logits into log s also forms the block metric of Eq. 6 for the
+ * blocks it holds, so the scores are not read back for it.  Arguments are those of the two calls;
+ * ws is one workspace of tca_workspace_bytes(prm, L, TCA_OP_SCORE_SELECT) bytes.  logscore, idx,
+ * h_out and t_out receive bit for bit what the two separate calls write.
+ */
+int tca_score_select(const tca_params* prm, const void* q_last, const void* K, int64_t L,
+                     const int32_t* n_k, int32_t nK, double* logscore, int32_t* idx,
+                     const int64_t* offsets_dev, double* h_out, int32_t* t_out,
+                     void* ws, size_t ws_bytes, void* stream);
 
 /* REQUIRED once after filling the descriptor and before any other call that takes it:
  * uploads the host mirror of `cache` (seg_start, global_cap, n_global, tail_head, n_tail,
@@ -332,6 +367,18 @@ int tca_attn_decode_static(const tca_params* prm, const void* q, const tca_cache
  * array has been cleared and the entry point can be used again.  Performs no allocation.  (No
  * counterpart in the paper.) */
 int tca_decode_static_status(void* stream);
+
+/*
+ * Range-checked build only (tca_build_info() & TCA_BUILD_DEBUG_BOUNDS; in the normal build this
+ * always returns TCA_OK).  tca_compact_kv and tca_cache_append take no workspace, so their range
+ * checks record a failure in the reserved state word of the unit concerned.  This call synchronises
+ * `stream`, reads the state words back and returns TCA_ERR_BOUNDS for the first unit whose word is
+ * set, with detail[0] = unit, detail[1] = which check (1 selected index, 2 block count, 3 ring
+ * slot, 4 cache row, 5 global region full), detail[2] = the offending value; detail HOST [3],
+ * optional.  The checked kernels skip the access that failed its test, so no build touches memory
+ * outside the buffers it was given.  tca_cache_init clears the words.
+ */
+int tca_cache_status(const tca_cache_desc* cache, void* stream, int64_t* detail);
 
 /* Synchronise `stream` and read the sticky status word at the start of a workspace: TCA_OK,
  * TCA_ERR_TIMEOUT if a bounded wait inside a kernel gave up, or (range-checked build)

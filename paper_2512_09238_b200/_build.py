@@ -4,6 +4,10 @@
 into an object file next to a stamp of its inputs and links them into
 ``paper_2512_09238_b200/libtca.so``.  Objects are rebuilt only when a source or header
 changed.  nvcc cross-compiles, so this works on a machine without a GPU.
+
+``build(debug_bounds=True)`` (``--debug-bounds`` on the command line) builds the range-checked
+variant ``libtca_dbg.so`` from the same sources with ``-DTCA_DEBUG_BOUNDS``: every index and
+offset a kernel reads from memory is compared with its range before use (see include/tca.h).
 """
 from __future__ import annotations
 
@@ -20,6 +24,7 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 BUILD = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libtca.so")
+LIB_DEBUG = os.path.join(PKG, "libtca_dbg.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -44,8 +49,8 @@ def _digest(paths) -> str:
     return h.hexdigest()
 
 
-def _compile(src: str, headers, verbose: bool, extra) -> str:
-    obj = os.path.join(BUILD, os.path.basename(src)[:-3] + ".o")
+def _compile(src: str, headers, verbose: bool, extra, build_dir: str = BUILD) -> str:
+    obj = os.path.join(build_dir, os.path.basename(src)[:-3] + ".o")
     stamp = obj + ".stamp"
     want = _digest([src, *headers]) + " ".join(extra)
     if os.path.exists(obj) and os.path.exists(stamp) and open(stamp).read() == want:
@@ -61,25 +66,29 @@ def _compile(src: str, headers, verbose: bool, extra) -> str:
     return obj
 
 
-def build(verbose: bool = False, ptxas_info: bool = False) -> str:
-    """Compile and link libtca.so; returns its path."""
-    os.makedirs(BUILD, exist_ok=True)
+def build(verbose: bool = False, ptxas_info: bool = False, debug_bounds: bool = False) -> str:
+    """Compile and link libtca.so (or, with debug_bounds, libtca_dbg.so); returns its path."""
+    build_dir = BUILD + "_dbg" if debug_bounds else BUILD
+    lib = LIB_DEBUG if debug_bounds else LIB
+    os.makedirs(build_dir, exist_ok=True)
     srcs = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers += [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE) if f.endswith(".h")]
     extra = ["-Xptxas", "-v"] if ptxas_info else []
+    if debug_bounds:
+        extra.append("-DTCA_DEBUG_BOUNDS")
     with cf.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
-        objs = list(ex.map(lambda s: _compile(s, headers, verbose or ptxas_info, extra), srcs))
+        objs = list(ex.map(lambda s: _compile(s, headers, verbose or ptxas_info, extra, build_dir), srcs))
     newest = max(os.path.getmtime(o) for o in objs)
-    if not os.path.exists(LIB) or os.path.getmtime(LIB) < newest:
-        cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
+    if not os.path.exists(lib) or os.path.getmtime(lib) < newest:
+        cmd = [_nvcc(), "-shared", "-o", lib, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
                "-Xcompiler", "-fPIC", "-lcuda"]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)
-            raise RuntimeError("link of libtca.so failed")
-    return LIB
+            raise RuntimeError(f"link of {os.path.basename(lib)} failed")
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(verbose=True, ptxas_info="--ptxas" in sys.argv))
+    print(build(verbose=True, ptxas_info="--ptxas" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

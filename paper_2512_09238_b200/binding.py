@@ -22,8 +22,11 @@ TCA_OK, TCA_ERR_INVALID_ARG, TCA_ERR_UNSUPPORTED, TCA_ERR_WORKSPACE = 0, -1, -2,
 TCA_ERR_CUDA, TCA_ERR_TIMEOUT, TCA_ERR_CAPACITY, TCA_ERR_SCRATCH_LIMIT, TCA_ERR_BOUNDS = -4, -5, -6, -7, -8
 TCA_DECODE_STATIC_SCRATCH_BYTES = 16 << 20
 TCA_F32, TCA_BF16 = 0, 1
-TCA_FLAG_PREFILL_SIMT = 1
-TCA_OP_SCORE, TCA_OP_SELECT, TCA_OP_COMPACT, TCA_OP_PREFILL, TCA_OP_DECODE, TCA_OP_APPEND, TCA_OP_CALIB = range(7)
+TCA_FLAG_PREFILL_SIMT, TCA_FLAG_ENTROPY_INDEX, TCA_FLAG_RANDOM_ORDER, TCA_FLAG_FLAT_TOPB = 1, 2, 4, 8
+TCA_FLAG_PREFILL_BAND_FIRST = 16
+TCA_BUILD_DEBUG_BOUNDS = 1
+(TCA_OP_SCORE, TCA_OP_SELECT, TCA_OP_COMPACT, TCA_OP_PREFILL, TCA_OP_DECODE, TCA_OP_APPEND, TCA_OP_CALIB,
+ TCA_OP_SCORE_SELECT) = range(8)
 TCA_STATE_WORDS = 8
 
 EXPORTS = (
@@ -31,7 +34,8 @@ EXPORTS = (
     "tca_select", "tca_cache_init", "tca_compact_kv", "tca_attn_prefill", "tca_attn_decode",
     "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
     "tca_calib_colmean", "tca_calib_score", "tca_calib_choose", "tca_calib_candidates",
-    "tca_decode_static_status", "tca_selftest_wait_expiry",
+    "tca_decode_static_status", "tca_selftest_wait_expiry", "tca_score_select", "tca_build_info",
+    "tca_cache_status",
 )
 
 
@@ -45,7 +49,7 @@ class tca_params(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("block", C.c_int32), ("window", C.c_int32),
                 ("alpha", C.c_float), ("sm_scale", C.c_float), ("dtype", C.c_int32),
-                ("flags", C.c_int32)]
+                ("flags", C.c_int32), ("seed", C.c_int32)]
 
 
 class tca_cache_desc(C.Structure):
@@ -59,53 +63,61 @@ class tca_cache_desc(C.Structure):
 _lib = None
 
 
+def load_library(path: str) -> C.CDLL:
+    """Load a build of the library from `path` and declare the argument types of its entry points."""
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with "
+                           "`python -m paper_2512_09238_b200._build` (needs nvcc)")
+    L = C.CDLL(path)
+    L.tca_strerror.restype = C.c_char_p
+    L.tca_strerror.argtypes = [C.c_int]
+    L.tca_version.restype = C.c_int
+    L.tca_workspace_bytes.restype = C.c_size_t
+    L.tca_workspace_bytes.argtypes = [C.POINTER(tca_params), C.c_int64, C.c_int]
+    L.tca_budget_resolve.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                     C.c_void_p, C.c_void_p]
+    P = C.POINTER(tca_params)
+    D = C.POINTER(tca_cache_desc)
+    vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+    L.tca_score.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
+    L.tca_select.argtypes = [P, vp, i64, vp, C.c_int32, vp, vp, vp, vp, vp, sz, vp]
+    L.tca_score_select.argtypes = [P, vp, vp, i64, vp, C.c_int32, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.tca_cache_init.argtypes = [P, D, vp]
+    L.tca_compact_kv.argtypes = [P, vp, vp, i64, vp, vp, vp, D, vp]
+    L.tca_attn_prefill.argtypes = [P, vp, vp, vp, i64, D, vp, vp, sz, vp]
+    L.tca_attn_prefill_rows.argtypes = [P, vp, vp, vp, i64, i64, i64, D, vp, vp, sz, vp]
+    L.tca_calib_colmean.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
+    L.tca_calib_score.argtypes = [P, vp, i64, vp, vp, vp, vp]
+    L.tca_calib_choose.argtypes = [vp, vp, C.c_int, C.c_double]
+    L.tca_calib_candidates.argtypes = [C.c_int, C.c_int, C.c_double, vp]
+    L.tca_attn_decode.argtypes = [P, vp, D, vp, vp, sz, vp]
+    L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
+    L.tca_ws_status.argtypes = [vp, vp]
+    L.tca_cache_status.argtypes = [D, vp, vp]
+    L.tca_attn_decode_static.argtypes = [P, vp, D, vp, vp]
+    L.tca_decode_static_status.argtypes = [vp]
+    L.tca_selftest_wait_expiry.argtypes = [vp, C.c_uint64, vp, vp]
+    L.tca_build_info.argtypes = []
+    for name in EXPORTS:
+        if name not in ("tca_strerror", "tca_workspace_bytes"):
+            getattr(L, name).restype = C.c_int
+    return L
+
+
 def lib() -> C.CDLL:
     """The loaded library; raises if it has not been built (no fallback exists)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
-                               "`python -m paper_2512_09238_b200._build` (needs nvcc)")
-        L = C.CDLL(LIB_PATH)
-        L.tca_strerror.restype = C.c_char_p
-        L.tca_strerror.argtypes = [C.c_int]
-        L.tca_version.restype = C.c_int
-        L.tca_workspace_bytes.restype = C.c_size_t
-        L.tca_workspace_bytes.argtypes = [C.POINTER(tca_params), C.c_int64, C.c_int]
-        L.tca_budget_resolve.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
-                                         C.c_void_p, C.c_void_p]
-        P = C.POINTER(tca_params)
-        D = C.POINTER(tca_cache_desc)
-        vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
-        L.tca_score.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
-        L.tca_select.argtypes = [P, vp, i64, vp, C.c_int32, vp, vp, vp, vp, vp, sz, vp]
-        L.tca_cache_init.argtypes = [P, D, vp]
-        L.tca_compact_kv.argtypes = [P, vp, vp, i64, vp, vp, vp, D, vp]
-        L.tca_attn_prefill.argtypes = [P, vp, vp, vp, i64, D, vp, vp, sz, vp]
-        L.tca_attn_prefill_rows.argtypes = [P, vp, vp, vp, i64, i64, i64, D, vp, vp, sz, vp]
-        L.tca_calib_colmean.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
-        L.tca_calib_score.argtypes = [P, vp, i64, vp, vp, vp, vp]
-        L.tca_calib_choose.argtypes = [vp, vp, C.c_int, C.c_double]
-        L.tca_calib_candidates.argtypes = [C.c_int, C.c_int, C.c_double, vp]
-        L.tca_attn_decode.argtypes = [P, vp, D, vp, vp, sz, vp]
-        L.tca_cache_append.argtypes = [P, D, vp, vp, vp, vp]
-        L.tca_ws_status.argtypes = [vp, vp]
-        L.tca_attn_decode_static.argtypes = [P, vp, D, vp, vp]
-        L.tca_decode_static_status.argtypes = [vp]
-        L.tca_selftest_wait_expiry.argtypes = [vp, C.c_uint64, vp, vp]
-        for name in EXPORTS:
-            if name not in ("tca_strerror", "tca_workspace_bytes"):
-                getattr(L, name).restype = C.c_int
-        _lib = L
+        _lib = load_library(LIB_PATH)
     return _lib
 
 
 # ----------------------------------------------------------------------------- helpers
 def make_params(batch, n_q_heads, n_kv_heads, head_dim, block, window, alpha=0.5, sm_scale=None,
-                dtype=TCA_BF16, flags=0) -> tca_params:
+                dtype=TCA_BF16, flags=0, seed=0) -> tca_params:
     if sm_scale is None:
         sm_scale = 1.0 / float(np.sqrt(head_dim))
-    return tca_params(batch, n_q_heads, n_kv_heads, head_dim, block, window, alpha, sm_scale, dtype, flags)
+    return tca_params(batch, n_q_heads, n_kv_heads, head_dim, block, window, alpha, sm_scale, dtype, flags, seed)
 
 
 def _dev(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -182,6 +194,24 @@ def tca_select(prm, logscore, L, n_k, idx, offsets_dev, h_out, t_out, ws, stream
     _check(lib().tca_select(C.byref(prm), _dev(logscore), L, _host(n_k, np.int32), n_k.shape[1], _dev(idx),
                             _dev(offsets_dev), _dev(h_out), _dev(t_out), *_ws_args(ws), _stream(stream)),
            "tca_select")
+
+
+def tca_score_select(prm, q_last, K, L, n_k, logscore, idx, offsets_dev, h_out, t_out, ws, stream=None) -> None:
+    n_k = np.ascontiguousarray(n_k, dtype=np.int32)
+    _check(lib().tca_score_select(C.byref(prm), _dev(q_last), _dev(K), L, _host(n_k, np.int32), n_k.shape[1],
+                                  _dev(logscore), _dev(idx), _dev(offsets_dev), _dev(h_out), _dev(t_out),
+                                  *_ws_args(ws), _stream(stream)), "tca_score_select")
+
+
+def tca_build_info() -> int:
+    return lib().tca_build_info()
+
+
+def tca_cache_status(cache: "Cache", stream=None):
+    """(status, detail) with detail = [unit, which check, offending value] when status is TCA_ERR_BOUNDS."""
+    detail = np.zeros(3, dtype=np.int64)
+    st = lib().tca_cache_status(C.byref(cache.desc), _stream(stream), detail.ctypes.data)
+    return st, detail
 
 
 def tca_cache_init(prm, cache: "Cache", stream=None) -> None:

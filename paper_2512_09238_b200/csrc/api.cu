@@ -18,7 +18,13 @@ int check_params(const tca_params* prm) {
   TCA_CHECK_ARG(prm->window >= 0);
   TCA_CHECK_ARG(prm->alpha >= 0.f && prm->alpha <= 1.f);
   TCA_CHECK_ARG(prm->sm_scale > 0.f && std::isfinite(prm->sm_scale));
-  TCA_CHECK_ARG((prm->flags & ~TCA_FLAG_PREFILL_SIMT) == 0);
+  constexpr int kKnownFlags = TCA_FLAG_PREFILL_SIMT | TCA_FLAG_ENTROPY_INDEX | TCA_FLAG_RANDOM_ORDER |
+                              TCA_FLAG_FLAT_TOPB | TCA_FLAG_PREFILL_BAND_FIRST;
+  TCA_CHECK_ARG((prm->flags & ~kKnownFlags) == 0);
+  {   // at most one selection variant
+    const int v = prm->flags & (TCA_FLAG_ENTROPY_INDEX | TCA_FLAG_RANDOM_ORDER | TCA_FLAG_FLAT_TOPB);
+    TCA_CHECK_ARG((v & (v - 1)) == 0);
+  }
   if (prm->dtype != TCA_F32 && prm->dtype != TCA_BF16) return TCA_ERR_UNSUPPORTED;
   if (prm->head_dim != 64 && prm->head_dim != 128) return TCA_ERR_UNSUPPORTED;
   if (!is_pow2(prm->block) || prm->block > kMaxBlock) return TCA_ERR_UNSUPPORTED;
@@ -45,9 +51,11 @@ SelectWs select_ws_layout(const tca_params* prm, int64_t L, void* ws) {
   const int64_t m = num_blocks(prm, L);
   size_t hkey_bytes = align_up(size_t(U) * (m > 0 ? m : 1) * sizeof(unsigned long long), 256);
   size_t t_bytes = align_up(size_t(U) * (m > 0 ? m : 1) * sizeof(int32_t), 256);
-  w.hkey = reinterpret_cast<unsigned long long*>(ws);
-  w.t = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(ws) + hkey_bytes);
-  w.bytes = hkey_bytes + t_bytes;
+  char* base = reinterpret_cast<char*>(ws);
+  w.status = reinterpret_cast<int*>(base);
+  w.hkey = reinterpret_cast<unsigned long long*>(base + 256);
+  w.t = reinterpret_cast<int32_t*>(base + 256 + hkey_bytes);
+  w.bytes = 256 + hkey_bytes + t_bytes;
   return w;
 }
 
@@ -83,7 +91,25 @@ const char* tca_strerror(int status) {
   }
 }
 
-int tca_version(void) { return 100; }
+int tca_version(void) { return 200; }
+
+int tca_build_info(void) { return kDebugBounds ? TCA_BUILD_DEBUG_BOUNDS : 0; }
+
+int tca_cache_status(const tca_cache_desc* c, void* stream, int64_t* detail) {
+  TCA_CHECK_ARG(c && c->state && c->n_units >= 1);
+  std::vector<int64_t> st(size_t(c->n_units) * TCA_STATE_WORDS);
+  TCA_CHECK_CUDA(cudaMemcpyAsync(st.data(), c->state, st.size() * sizeof(int64_t), cudaMemcpyDeviceToHost,
+                                 static_cast<cudaStream_t>(stream)));
+  TCA_CHECK_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  for (int64_t u = 0; u < c->n_units; ++u) {
+    const int64_t word = st[size_t(u) * TCA_STATE_WORDS + TCA_ST_RESERVED];
+    if (word != 0) {
+      if (detail) { detail[0] = u; detail[1] = int64_t(uint64_t(word) >> 56); detail[2] = word & 0x00FFFFFFFFFFFFFFll; }
+      return TCA_ERR_BOUNDS;
+    }
+  }
+  return TCA_OK;
+}
 
 int tca_budget_resolve(const double* p, int32_t n_kv_heads, int32_t nK, int64_t m,
                        int32_t* n_k, int64_t* n_sel, int32_t* tbar) {
@@ -140,6 +166,8 @@ size_t tca_workspace_bytes(const tca_params* prm, int64_t L, int op) {
     case TCA_OP_DECODE: return decode_ws_layout(prm, L, U, nullptr).bytes;
     case TCA_OP_APPEND: return 256;
     case TCA_OP_CALIB: return prm->dtype == TCA_BF16 ? calib_ws_bytes(prm, L) : 0;
+    case TCA_OP_SCORE_SELECT:
+      return align_up(score_ws_layout(prm, L, nullptr).bytes, 256) + select_ws_layout(prm, L, nullptr).bytes;
     default: return 0;
   }
 }

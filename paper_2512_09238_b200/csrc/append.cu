@@ -30,6 +30,15 @@ cache_append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, co
   const int64_t ring = seg + gcap;
   __syncthreads();  // every thread has read the state before anyone updates it
 
+  if constexpr (kDebugBounds) {
+    // the state words this kernel indexes with: ring position and fill, and room for a kept block
+    const bool bad_ring = tail_head < 0 || tail_head >= tail_cap || n_tail < 0 || n_tail >= tail_cap;
+    const bool bad_room = (n_tail + 1 >= int64_t(window) + b) && (t_keep < 0 || t_keep > b || n_global + t_keep > gcap);
+    if (bad_ring || bad_room) {
+      if (tid == 0) report_bounds_state(st, bad_ring ? kBoundsRingSlot : kBoundsGlobalRegion, bad_ring ? tail_head : n_global);
+      return;
+    }
+  }
   // ---- append
   {
     const int64_t slot = (tail_head + n_tail) % tail_cap;

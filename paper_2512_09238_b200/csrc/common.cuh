@@ -11,6 +11,19 @@ namespace tca {
 
 constexpr int kStatusTimeout = 1;  // values of a workspace's status word
 constexpr int kStatusBounds = 2;
+
+// Range-checked build (-DTCA_DEBUG_BOUNDS): every index or offset that a kernel takes from memory
+// (selected token indices, per-block counts, ring slots, cache rows) is compared with its range
+// before it is used; an access that fails the test is skipped and the first failure is recorded
+// where the host can read it (word 0 of the workspace, or the reserved state word of the unit for
+// the calls that take no workspace).  Nothing traps.  In the normal build the checks compile away.
+#ifdef TCA_DEBUG_BOUNDS
+constexpr bool kDebugBounds = true;
+#else
+constexpr bool kDebugBounds = false;
+#endif
+enum { kBoundsSelectedIndex = 1, kBoundsBlockCount = 2, kBoundsRingSlot = 3, kBoundsCacheRow = 4,
+       kBoundsGlobalRegion = 5 };
 constexpr int kMaxGroup = 8;    // query heads per KV head
 constexpr int kMaxBlock = 128;  // b
 
@@ -56,8 +69,9 @@ struct ScoreWs {
 };
 ScoreWs score_ws_layout(const tca_params* prm, int64_t L, void* ws);
 
-// select: hkey [U][m] uint64, t [U][m] int32.
+// select: a 256-byte header (word 0: status, range-checked build), hkey [U][m] uint64, t [U][m] int32.
 struct SelectWs {
+  int* status;
   unsigned long long* hkey;
   int32_t* t;
   size_t bytes;
@@ -110,6 +124,22 @@ template <>
 struct Elt<__nv_bfloat16> {
   static constexpr int kDtype = TCA_BF16;
 };
+
+// Record a failed range check in a workspace header: word 0 = kStatusBounds, word 1 = which check,
+// bytes 8..15 = the offending value.  Only the first failure is kept.
+__device__ __forceinline__ void report_bounds_ws(int* status, int which, long long value) {
+  if (atomicCAS(status, 0, kStatusBounds) == 0) {
+    status[1] = which;
+    reinterpret_cast<long long*>(status)[1] = value;
+  }
+}
+// The same for the calls without a workspace: the unit's reserved state word takes
+// (which << 56) | (value & 2^56 - 1); zero means "no failure".
+__device__ __forceinline__ void report_bounds_state(int64_t* unit_state, int which, long long value) {
+  const unsigned long long word = (static_cast<unsigned long long>(which) << 56) |
+                                  (static_cast<unsigned long long>(value) & 0x00FFFFFFFFFFFFFFull);
+  atomicCAS(reinterpret_cast<unsigned long long*>(unit_state + TCA_ST_RESERVED), 0ull, word);
+}
 
 // Order-preserving map double -> uint64 (a < b  <=>  key(a) < key(b); -0 < +0).
 __device__ __forceinline__ unsigned long long ordered_key(double x) {

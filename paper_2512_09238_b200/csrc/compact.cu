@@ -51,6 +51,13 @@ compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t
         const int piece = int(p & (pieces_per_row - 1));
         const int64_t s = (r < n_sel) ? int64_t(idx[off + r]) : tail_begin + (r - n_sel);
         const int64_t drow = (r < n_sel) ? seg + r : seg + gcap + (r - n_sel);
+        if constexpr (kDebugBounds) {
+          // a selected index must name a candidate token, and its row must fit the global region
+          if (r < n_sel && (s < 0 || s >= tail_begin || r >= gcap)) {
+            if (piece == 0) report_bounds_state(st, kBoundsSelectedIndex, s);
+            continue;   // skip the access: dst[i] stays -1
+          }
+        }
         src[i] = int32_t(s);
         lead[i] = piece == 0;
         dst[i] = drow * pieces_per_row + piece;

@@ -107,6 +107,14 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
             while (done < cnt) {   // at most three physically contiguous runs
               const int64_t r = row0 + trow + done;
               const int run = int(uv.run(r, cnt - done));
+              if constexpr (kDebugBounds) {
+                const int64_t y = uv.phys(r);
+                if (run <= 0 || y < uv.seg || y + run > uv.seg + uv.gcap + uv.tail_cap) {
+                  report_bounds_ws(status, kBoundsCacheRow, y);
+                  *abort_flag = 1;   // the consumers leave their waits; nothing is copied
+                  return;
+                }
+              }
               bulk_copy_g2s(dst + size_t(done) * D * sizeof(T), src + size_t(uv.phys(r)) * D,
                             uint32_t(run) * D * sizeof(T), &ring.full[n % kStages]);
               done += run;
@@ -251,7 +259,7 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
     consumer_sync(kConsumers);   // xs is rewritten by the next round
   }
   if (*abort_flag) {   // uniform after the barrier above: some wait gave up, the result is not valid
-    if (tid == 0) atomicExch(status, 1);
+    if (tid == 0) atomicCAS(status, 0, kStatusTimeout);   // keeps an earlier, more specific code
     return;
   }
 

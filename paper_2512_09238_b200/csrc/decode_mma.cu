@@ -107,6 +107,14 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         const int64_t r = row0 + done;
         const int cnt = int(min(int64_t(kMmaTileRows), uv.run(r, n_rows - done)));
         const int y = int(uv.phys(r));
+        if constexpr (kDebugBounds) {
+          // the tile must lie inside the unit's segment (the tensor map bounds the whole cache only)
+          if (y < uv.seg || int64_t(y) + cnt > uv.seg + uv.gcap + uv.tail_cap) {
+            report_bounds_ws(status, kBoundsCacheRow, y);
+            *abort_flag = 1;   // the consumers leave their waits; nothing is copied
+            return;
+          }
+        }
         for (int kv = 0; kv < 2; ++kv, ++n) {
           if (!ring.acquire(n, uint32_t(Ring::kTileBytes), abort_flag)) return;
           uint8_t* dst = ring_buf + (n % kStages) * Ring::kTileBytes;
@@ -232,7 +240,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   }
   consumer_sync(kMmaConsumers);
   if (*abort_flag) {
-    if (tid == 0) atomicExch(status, 1);
+    if (tid == 0) atomicCAS(status, 0, kStatusTimeout);   // keeps an earlier, more specific code
     return;
   }
   float* out = partial + size_t(base_slot + part_idx) * G * (D + 2);

@@ -70,7 +70,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 // the shared memory they target is handed back.  (TMEM is freed by the caller, as on the normal
 // path.)  Must be reached by every thread of the CTA.
 __device__ __forceinline__ void abort_teardown(int* status, int tid) {
-  if (tid == 0) atomicExch(status, 1);
+  if (tid == 0) atomicCAS(status, 0, 1);   // 1 = a wait gave up; an earlier code is kept
   for (int i = 0; i < 64; ++i) __nanosleep(2000);
   __syncthreads();
 }

@@ -7,8 +7,12 @@
 // blocking, queries from shared memory), see the kernel.  Each CTA also leaves a
 // (max, sum-exp) partial per head.
 // Pass 2 (score_finalize_kernel) merges the partials into each head's log-sum-exp and
-// turns logits into  log( (1/G) * sum_g softmax_g[j] ).
+// turns logits into  log( (1/G) * sum_g softmax_g[j] ).  When asked to (tca_score_select), its
+// CTAs, which each hold 1024 consecutive log-scores = whole blocks of b tokens, also form the
+// block metric h_j of Eq. 6 for those blocks, so that the selection does not read the scores
+// back for it.
 #include "common.cuh"
+#include "select_common.cuh"
 
 namespace tca {
 namespace {
@@ -179,13 +183,16 @@ score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64
   }
 }
 
+constexpr int kFinalizeRows = 1024;   // log-scores per CTA of the second pass: a multiple of every block size b <= 128
+
 template <int G>
 __global__ void __launch_bounds__(kThreads)
 score_finalize_kernel(const double* __restrict__ logits, const double* __restrict__ partials, int n_chunks,
-                      int64_t L, double* __restrict__ logscore, int rows_per_cta) {
+                      int64_t L, double* __restrict__ logscore, MetricOut mo) {
   const int u = blockIdx.y;
   const int tid = threadIdx.x;
   __shared__ double lse[G];
+  __shared__ double ls_s[kFinalizeRows];   // this CTA's log-scores, for the fused block metric
   // log-sum-exp of every head of the group from the per-chunk partials (warp g does head g)
   {
     const int warp = tid >> 5, lane = tid & 31;
@@ -206,8 +213,8 @@ score_finalize_kernel(const double* __restrict__ logits, const double* __restric
   __syncthreads();
   const double log_g = log(double(G));
   const double* lu = logits + size_t(u) * G * L;
-  const int64_t j0 = int64_t(blockIdx.x) * rows_per_cta;
-  const int64_t j1 = min(j0 + int64_t(rows_per_cta), L);
+  const int64_t j0 = int64_t(blockIdx.x) * kFinalizeRows;
+  const int64_t j1 = min(j0 + int64_t(kFinalizeRows), L);
   for (int64_t j = j0 + tid; j < j1; j += kThreads) {
     double y[G];
     double top = -1.0e308;
@@ -216,20 +223,38 @@ score_finalize_kernel(const double* __restrict__ logits, const double* __restric
       y[g] = lu[size_t(g) * L + j] - lse[g];
       top = fmax(top, y[g]);
     }
+    double out;
     if (G == 1) {
-      logscore[size_t(u) * L + j] = y[0];
+      out = y[0];
     } else {
       float sum = 0.f;
 #pragma unroll
       for (int g = 0; g < G; ++g) sum += expf(float(y[g] - top));
-      logscore[size_t(u) * L + j] = top + double(logf(sum)) - log_g;
+      out = top + double(logf(sum)) - log_g;
+    }
+    logscore[size_t(u) * L + j] = out;
+    ls_s[j - j0] = out;
+  }
+  if (mo.hkey == nullptr) return;
+  // Fused tail: h_j for the blocks that lie in [j0, j1); blocks j >= m belong to the always-kept
+  // tail and have no metric.  Same arithmetic as block_metric_kernel on the same doubles.
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31;
+  const int jb0 = int(j0 / mo.b);
+  for (int i = warp; i < kFinalizeRows / mo.b; i += kThreads / 32) {
+    const int jb = jb0 + i;
+    if (jb >= mo.m) break;
+    const double h = block_metric_warp(ls_s + i * mo.b, mo.b, mo.alpha, mo.mode, lane);
+    if (lane == 0) {
+      mo.hkey[size_t(u) * mo.m + jb] = ordered_key(h);
+      if (mo.h_out) mo.h_out[size_t(u) * mo.m + jb] = h;
     }
   }
 }
 
 template <typename T, int D, int G>
 int launch_score(const tca_params* prm, const void* q_last, const void* K, int64_t L, double* logscore,
-                 const ScoreWs& ws, cudaStream_t stream) {
+                 const ScoreWs& ws, const MetricOut& mo, cudaStream_t stream) {
   const int U = prm->batch * prm->n_kv_heads;
   dim3 grid1(unsigned(ws.n_chunks), unsigned(U));
   score_logits_kernel<T, D, G><<<grid1, kLogitThreads, 0, stream>>>(
@@ -237,30 +262,50 @@ int launch_score(const tca_params* prm, const void* q_last, const void* K, int64
       ws.partials, int(ws.n_chunks));
   int st = check_launch();
   if (st != TCA_OK) return st;
-  const int rows_per_cta = 1024;
-  dim3 grid2(unsigned((L + rows_per_cta - 1) / rows_per_cta), unsigned(U));
+  dim3 grid2(unsigned((L + kFinalizeRows - 1) / kFinalizeRows), unsigned(U));
   score_finalize_kernel<G><<<grid2, kThreads, 0, stream>>>(ws.logits, ws.partials, int(ws.n_chunks), L,
-                                                           logscore, rows_per_cta);
+                                                           logscore, mo);
   return check_launch();
 }
 
 template <typename T, int D>
 int dispatch_group(int G, const tca_params* prm, const void* q_last, const void* K, int64_t L,
-                   double* logscore, const ScoreWs& ws, cudaStream_t stream) {
+                   double* logscore, const ScoreWs& ws, const MetricOut& mo, cudaStream_t stream) {
   switch (G) {
-    case 1: return launch_score<T, D, 1>(prm, q_last, K, L, logscore, ws, stream);
-    case 2: return launch_score<T, D, 2>(prm, q_last, K, L, logscore, ws, stream);
-    case 3: return launch_score<T, D, 3>(prm, q_last, K, L, logscore, ws, stream);
-    case 4: return launch_score<T, D, 4>(prm, q_last, K, L, logscore, ws, stream);
-    case 5: return launch_score<T, D, 5>(prm, q_last, K, L, logscore, ws, stream);
-    case 6: return launch_score<T, D, 6>(prm, q_last, K, L, logscore, ws, stream);
-    case 7: return launch_score<T, D, 7>(prm, q_last, K, L, logscore, ws, stream);
-    case 8: return launch_score<T, D, 8>(prm, q_last, K, L, logscore, ws, stream);
+    case 1: return launch_score<T, D, 1>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 2: return launch_score<T, D, 2>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 3: return launch_score<T, D, 3>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 4: return launch_score<T, D, 4>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 5: return launch_score<T, D, 5>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 6: return launch_score<T, D, 6>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 7: return launch_score<T, D, 7>(prm, q_last, K, L, logscore, ws, mo, stream);
+    case 8: return launch_score<T, D, 8>(prm, q_last, K, L, logscore, ws, mo, stream);
     default: return TCA_ERR_UNSUPPORTED;
   }
 }
 
 }  // namespace
+
+// tca_score proper; `fused.hkey != nullptr` also leaves the block metric of Eq. 6 there.
+int score_impl(const tca_params* prm, const void* q_last, const void* K, int64_t L, double* logscore, void* ws,
+               size_t ws_bytes, const MetricOut& fused, cudaStream_t s) {
+  TCA_CHECK_ARG(q_last && K && logscore && ws);
+  TCA_CHECK_ARG(L >= 1 && L < (int64_t(1) << 31));
+  TCA_CHECK_ARG(aligned(q_last, 16) && aligned(K, 16) && aligned(logscore, 8) && aligned(ws, 256));
+  const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
+  TCA_CHECK_ARG(U <= 65535);
+  ScoreWs lay = score_ws_layout(prm, L, ws);
+  if (ws_bytes < lay.bytes) return TCA_ERR_WORKSPACE;
+  if (fused.hkey && kFinalizeRows % fused.b != 0) return TCA_ERR_UNSUPPORTED;
+  const int G = prm->n_q_heads / prm->n_kv_heads;
+  if (prm->dtype == TCA_BF16) {
+    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q_last, K, L, logscore, lay, fused, s);
+    return dispatch_group<__nv_bfloat16, 64>(G, prm, q_last, K, L, logscore, lay, fused, s);
+  }
+  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q_last, K, L, logscore, lay, fused, s);
+  return dispatch_group<float, 64>(G, prm, q_last, K, L, logscore, lay, fused, s);
+}
+
 }  // namespace tca
 
 using namespace tca;
@@ -269,19 +314,6 @@ extern "C" int tca_score(const tca_params* prm, const void* q_last, const void* 
                          double* logscore, void* ws, size_t ws_bytes, void* stream) {
   int st = check_params(prm);
   if (st != TCA_OK) return st;
-  TCA_CHECK_ARG(q_last && K && logscore && ws);
-  TCA_CHECK_ARG(L >= 1 && L < (int64_t(1) << 31));
-  TCA_CHECK_ARG(aligned(q_last, 16) && aligned(K, 16) && aligned(logscore, 8) && aligned(ws, 256));
-  const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
-  TCA_CHECK_ARG(U <= 65535);
-  ScoreWs lay = score_ws_layout(prm, L, ws);
-  if (ws_bytes < lay.bytes) return TCA_ERR_WORKSPACE;
-  const int G = prm->n_q_heads / prm->n_kv_heads;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (prm->dtype == TCA_BF16) {
-    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q_last, K, L, logscore, lay, s);
-    return dispatch_group<__nv_bfloat16, 64>(G, prm, q_last, K, L, logscore, lay, s);
-  }
-  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q_last, K, L, logscore, lay, s);
-  return dispatch_group<float, 64>(G, prm, q_last, K, L, logscore, lay, s);
+  const MetricOut none{nullptr, nullptr, 0, 1, 0, 0.0};
+  return score_impl(prm, q_last, K, L, logscore, ws, ws_bytes, none, static_cast<cudaStream_t>(stream));
 }

@@ -1,6 +1,6 @@
 // Host-side encoding of TMA tensor maps for row-major bf16 matrices (128-byte swizzle, boxes of
-// 128 rows x 64 columns), through the driver entry point so that the library does not link
-// against libcuda.
+// 128 rows x 64 columns).  The encoder is looked up through the runtime's driver entry point
+// query, so that its version always matches the driver that is loaded.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>

@@ -31,9 +31,9 @@ def from_device(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def params_for(wl: I.Workload, flags: int = 0) -> B.tca_params:
+def params_for(wl: I.Workload, flags: int = 0, seed: int = 0) -> B.tca_params:
     return B.make_params(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.block, wl.window,
-                         alpha=wl.alpha, dtype=B.TCA_BF16 if wl.dtype == "bf16" else B.TCA_F32, flags=flags)
+                         alpha=wl.alpha, dtype=B.TCA_BF16 if wl.dtype == "bf16" else B.TCA_F32, flags=flags, seed=seed)
 
 
 def scale_of(wl: I.Workload) -> float:
@@ -60,10 +60,11 @@ class DeviceRun:
 
 
 def gpu_select_compact(wl: I.Workload, data: Dict[str, np.ndarray], p: np.ndarray, L: Optional[int] = None,
-                       extra_blocks: int = 0, flags: int = 0) -> DeviceRun:
-    """score -> select -> compact on the GPU for the first L tokens of `data`."""
+                       extra_blocks: int = 0, flags: int = 0, seed: int = 0, fused: bool = False) -> DeviceRun:
+    """score -> select -> compact on the GPU for the first L tokens of `data` (fused: score and
+    select through the single tca_score_select call)."""
     L = wl.L if L is None else L
-    prm = params_for(wl, flags)
+    prm = params_for(wl, flags, seed)
     U = wl.batch * wl.n_kv_heads
     dev = {k: to_device(np.ascontiguousarray(v[:, :, :L]), wl.dtype) for k, v in data.items()}
     m = max(0, (L - wl.window) // wl.block)
@@ -74,11 +75,19 @@ def gpu_select_compact(wl: I.Workload, data: Dict[str, np.ndarray], p: np.ndarra
     offsets_dev = torch.from_numpy(offsets).cuda()
     logscore = torch.empty(U, L, dtype=torch.float64, device="cuda")
     q_last = dev["q"][:, :, L - 1, :].contiguous()
-    B.tca_score(prm, q_last, dev["k"], L, logscore, B.alloc_workspace(prm, L, B.TCA_OP_SCORE))
     idx = torch.full((max(1, int(offsets[-1])),), -1, dtype=torch.int32, device="cuda")
     h = torch.zeros(U, max(1, m), dtype=torch.float64, device="cuda")
     t = torch.zeros(U, max(1, m), dtype=torch.int32, device="cuda")
-    B.tca_select(prm, logscore, L, n_k, idx, offsets_dev, h, t, B.alloc_workspace(prm, L, B.TCA_OP_SELECT))
+    if fused:
+        ws = B.alloc_workspace(prm, L, B.TCA_OP_SCORE_SELECT)
+        B.tca_score_select(prm, q_last, dev["k"], L, n_k, logscore, idx, offsets_dev, h, t, ws)
+        assert B.tca_ws_status(ws[B.tca_workspace_bytes(prm, L, B.TCA_OP_SCORE_SELECT)
+                                  - B.tca_workspace_bytes(prm, L, B.TCA_OP_SELECT):]) == B.TCA_OK
+    else:
+        B.tca_score(prm, q_last, dev["k"], L, logscore, B.alloc_workspace(prm, L, B.TCA_OP_SCORE))
+        ws = B.alloc_workspace(prm, L, B.TCA_OP_SELECT)
+        B.tca_select(prm, logscore, L, n_k, idx, offsets_dev, h, t, ws)
+        assert B.tca_ws_status(ws) == B.TCA_OK
     tk = np.tile(tbar, wl.batch).astype(np.int64)
     cache = B.Cache(prm, per_unit + extra_blocks * tk, wl.window + wl.block, tk)
     B.tca_compact_kv(prm, dev["k"], dev["v"], L, idx, offsets_dev, offsets, cache)
@@ -162,3 +171,16 @@ def sample_rows(L: int, w: int, b: int, n_random: int, seed: int) -> List[int]:
     rng = np.random.default_rng(seed)
     rows.update(int(x) for x in rng.integers(0, L, size=n_random))
     return sorted(rows)
+
+
+def compare_flat_selection(log_s: np.ndarray, gpu_S: np.ndarray, n_keep: int, n_candidates: int) -> int:
+    """The 1e-5 rule for the flat top-B variant: the GPU's set equals the oracle's, or differs only
+    in tokens whose oracle score is within 1e-5 of the n_keep-th largest.  Returns accepted swaps."""
+    want = O.select_tokens_flat(log_s, n_keep, n_candidates)
+    assert np.all(np.diff(gpu_S) > 0) and len(gpu_S) == n_keep and (n_keep == 0 or gpu_S.max() < n_candidates)
+    if np.array_equal(gpu_S, want):
+        return 0
+    boundary = np.sort(log_s[:n_candidates])[::-1][n_keep - 1]
+    diff = np.setxor1d(gpu_S, want)
+    assert np.all(np.abs(log_s[diff] - boundary) < SEL_TOL), "flat top-B kept the wrong tokens"
+    return len(diff) // 2

@@ -366,6 +366,80 @@ def test_append_compress_and_decode_steps(name, steps):
         np.testing.assert_array_equal(Kc[run.cache.unit_rows(u)], data["k"][s, h, c.positions()].view(Kc.dtype))
 
 
+@pytest.mark.parametrize("name", ["config1", "bf16_gqa4", "bf16_g7", "f32_g3_b1"])
+def test_fused_score_select_is_bit_identical_to_the_two_calls(runs, name):
+    """tca_score_select (the block metric formed in the tail of the score kernel) against
+    tca_score + tca_select: same log s, h, t and index set, bit for bit."""
+    wl, data, p, run, oracle = runs(name)
+    fused = H.gpu_select_compact(wl, data, p, fused=True)
+    assert torch.equal(fused.logscore.view(torch.int64), run.logscore.view(torch.int64))
+    assert torch.equal(fused.h.view(torch.int64), run.h.view(torch.int64))
+    assert torch.equal(fused.t, run.t) and torch.equal(fused.idx, run.idx)
+    assert torch.equal(fused.cache.pos, run.cache.pos)
+
+
+@pytest.mark.parametrize("name", ["config1", "bf16_gqa4", "bf16_d64_g2", "bf16_g7"])
+@pytest.mark.parametrize("variant", ["entropy", "random", "flat"])
+def test_selection_variants_match_their_oracles(name, variant):
+    """The ablation variants (entropy concentration index, seeded random block order) and the flat
+    top-B as modes of tca_select, through score -> select -> compact -> prefill, each against the
+    oracle's variant; the fused call takes the same path for the entropy index."""
+    wl = SMALL[name]
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    flags = {"entropy": B.TCA_FLAG_ENTROPY_INDEX, "random": B.TCA_FLAG_RANDOM_ORDER, "flat": B.TCA_FLAG_FLAT_TOPB}[variant]
+    seed = 12345
+    run = H.gpu_select_compact(wl, data, p, flags=flags, seed=seed, fused=(variant == "entropy"))
+    idx, t, hh = run.idx.cpu().numpy(), run.t.cpu().numpy(), run.h.cpu().numpy()
+    G, scale = wl.group, H.scale_of(wl)
+    differs = 0
+    for s_ in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            u = s_ * wl.n_kv_heads + h
+            K = I.widen(data["k"][s_, h, :wl.L])
+            q_last = I.widen(data["q"][s_, h * G:(h + 1) * G, wl.L - 1])
+            res = O.select_head_variant(q_last, K, p[h], wl.block, wl.window, float(np.float32(wl.alpha)), scale,
+                                        variant, seed=seed, unit=u)
+            S = idx[run.offsets[u]:run.offsets[u + 1]].astype(np.int64)
+            if variant == "flat":
+                assert H.compare_flat_selection(res["log_s"], S, int(run.n_sel[h]), res["m"] * wl.block) <= 1
+            else:
+                if variant == "random":
+                    np.testing.assert_array_equal(hh[u, :res["m"]], res["h"])          # the hash keys, exactly
+                else:
+                    np.testing.assert_allclose(hh[u, :res["m"]], res["h"], rtol=2e-6, atol=1e-12)
+                assert H.compare_selection(res, S, t[u, :res["m"]], wl.block) <= 1
+            base = O.select_head(q_last, K, p[h], wl.block, wl.window, float(np.float32(wl.alpha)), scale)
+            differs += not np.array_equal(base["S"], S)
+    assert differs > 0 or variant == "entropy"       # a variant that changed nothing would test nothing
+    # the rest of the path does not care how the set was chosen
+    out = H.from_device(H.gpu_prefill(run))
+    u = wl.batch * wl.n_kv_heads - 1
+    s_, h = divmod(u, wl.n_kv_heads)
+    T = _oracle_T(run, wl, u)
+    rows = H.sample_rows(wl.L, wl.window, wl.block, 16, seed=3)
+    want = O.attention_rows(I.widen(data["q"][s_, h * G, :wl.L]), I.widen(data["k"][s_, h, :wl.L]),
+                            I.widen(data["v"][s_, h, :wl.L]), T, wl.window, scale, rows)
+    H.check_attention(out[s_, h * G][rows], want, wl.dtype, f"{name} {variant}")
+
+
+def test_flat_top_b_at_a_size_with_many_radix_passes_and_ties():
+    """The flat variant's radix select over tens of thousands of candidates, with exact ties at the
+    threshold (scores injected directly): equal keys go to the lower position."""
+    L, b, w = 40000, 64, 1088
+    m = (L - w) // b
+    prm = B.make_params(1, 1, 1, 64, b, w, dtype=B.TCA_F32, flags=B.TCA_FLAG_FLAT_TOPB)
+    rng = np.random.default_rng(77)
+    ls = np.round(rng.standard_normal(L) * 3.0, 2)               # two decimals: thousands of exact ties
+    logscore = torch.from_numpy(ls).cuda().reshape(1, L)
+    pk = np.zeros((1, 7)); pk[0, 2] = 1.0                        # 4 tokens per block
+    n_k, n_sel, _ = B.tca_budget_resolve(pk, m)
+    offsets = torch.tensor([0, int(n_sel[0])], dtype=torch.int64, device="cuda")
+    idx = torch.full((int(n_sel[0]),), -1, dtype=torch.int32, device="cuda")
+    B.tca_select(prm, logscore, L, n_k, idx, offsets, None, None, B.alloc_workspace(prm, L, B.TCA_OP_SELECT))
+    np.testing.assert_array_equal(idx.cpu().numpy(), O.select_tokens_flat(ls, int(n_sel[0]), m * b))
+
+
 def test_capacity_and_workspace_errors():
     wl = SMALL["bf16_d64_g2"]
     data = I.generate(wl)

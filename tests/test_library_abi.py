@@ -28,12 +28,13 @@ def test_every_declared_symbol_is_exported():
     cdll = ctypes.CDLL(B.LIB_PATH)
     for name in declared:
         assert hasattr(cdll, name), f"{name} is declared but not exported"
-    assert B.tca_version() >= 100
+    assert B.tca_version() >= 200
+    assert B.tca_build_info() == 0                       # the default build carries no range checks
     assert B.tca_strerror(0) == "ok" and "workspace" in B.tca_strerror(B.TCA_ERR_WORKSPACE)
 
 
 def test_struct_layouts_match_the_header():
-    assert ctypes.sizeof(B.tca_params) == 40
+    assert ctypes.sizeof(B.tca_params) == 44
     assert ctypes.sizeof(B.tca_cache_desc) == 14 * 8
 
 
@@ -108,6 +109,18 @@ def test_static_decode_limit_formula_is_the_workspace_size():
         U, G = batch * hkv, hq // hkv
         want = 256 + up((rows // 256 + 2 * U + 1) * G * (d + 2) * 4)
         assert B.tca_workspace_bytes(prm, rows, B.TCA_OP_DECODE) == want
+
+
+def test_selection_variant_flags_are_validated():
+    ok = dict(batch=1, n_q_heads=8, n_kv_heads=8, head_dim=64, block=32, window=128, dtype=B.TCA_F32)
+    for flags in (0, B.TCA_FLAG_ENTROPY_INDEX, B.TCA_FLAG_RANDOM_ORDER, B.TCA_FLAG_FLAT_TOPB,
+                  B.TCA_FLAG_ENTROPY_INDEX | B.TCA_FLAG_PREFILL_SIMT, B.TCA_FLAG_PREFILL_BAND_FIRST):
+        assert B.tca_workspace_bytes(B.make_params(flags=flags, **ok), 2048, B.TCA_OP_SELECT) > 0
+    for flags in (B.TCA_FLAG_ENTROPY_INDEX | B.TCA_FLAG_FLAT_TOPB, B.TCA_FLAG_RANDOM_ORDER | B.TCA_FLAG_ENTROPY_INDEX, 32, 1 << 20):
+        assert B.tca_workspace_bytes(B.make_params(flags=flags, **ok), 2048, B.TCA_OP_SELECT) == 0
+    prm = B.make_params(**ok)
+    both = B.tca_workspace_bytes(prm, 2048, B.TCA_OP_SCORE_SELECT)
+    assert both >= B.tca_workspace_bytes(prm, 2048, B.TCA_OP_SCORE) + B.tca_workspace_bytes(prm, 2048, B.TCA_OP_SELECT)
 
 
 def test_workspace_sizes_scale_as_documented():
