@@ -411,6 +411,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the 100 %-budget comparison run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="config5: skip the five-budget sweep")
     ap.add_argument("--no-calibration", action="store_true", help="skip the offline calibration (Algorithm 1) leg")
     args = ap.parse_args()
 
@@ -555,6 +556,29 @@ def main():
                                  "kv_rows_retained_vs_dense": work["retained_fraction"]}
         del pipe
         torch.cuda.empty_cache()
+        pipe = main_pipe
+
+    if wl.name == "config5" and not args.no_sweep:
+        # the budget sweep of this configuration in one invocation: 5, 10, 25, 50 and 100 % of the candidates,
+        # each with its own prefill and its own decode steps, timed like the main run
+        main_pipe, sweep = pipe, {}
+        for frac in (0.05, 0.10, 0.25, 0.50, 1.0):
+            wl_f = wl_rank.scaled(budget=("fixed", frac))
+            pipe = Pipeline(wl_f, data, I.budget_table(wl_f), torch, B, host_io=False)
+            _, st_f, _ = timed(host_io=False)
+            assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK and B.tca_ws_status(pipe.ws_decode) == B.TCA_OK
+            wk = pipe.algorithmic_work()
+            pf = st_f["score_select"] + st_f["compact"] + st_f["prefill"]
+            dus = st_f["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None
+            sweep[f"{frac:.2f}"] = {
+                "prefill_ms": pf, "prefill_tok_s": job_throughput(world, wl.batch, wl.L, pf),
+                "attention_tflops": wk["prefill_flops"] / (st_f["prefill"] * 1e-3) / 1e12,
+                "decode_us_per_step": dus,
+                "decode_frac_of_measured_hbm": (wk["decode_bytes_per_step"] / (dus * 1e-6) / 1e9 / hbm) if dus else None,
+                "retained_fraction": wk["retained_fraction"]}
+            del pipe
+            torch.cuda.empty_cache()
+        out["budget_sweep"] = sweep
         pipe = main_pipe
 
     if not args.no_e2e:
