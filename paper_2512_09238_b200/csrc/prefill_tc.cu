@@ -17,8 +17,9 @@
 // programmatic dependent launch, starts on the band while those kernels are still running
 // and waits for them (griddepcontrol.wait) only where it first touches the cache.
 //
-// Warp roles (384 threads = 3 warpgroups): warp 0 = TMA producer (lane 0) and geometry (lane 1),
-// warp 1 = MMA issuer, warps 2-3 idle; warps 4-7 / 8-11 = softmax of head 0 / head 1 (one thread per
+// Warp roles (384 threads = 3 warpgroups): warp 0 = TMA producer (one lane), warp 1 = MMA issuer,
+// warp 2 = geometry of the global range (a warp-wide search at the start), warp 3 idle;
+// warps 4-7 / 8-11 = softmax of head 0 / head 1 (one thread per
 // query row = one TMEM lane).  The first warpgroup hands most of its registers to the other two
 // (setmaxnreg), so that a softmax thread can hold its row of 128 scores without spilling.
 // TMEM (512 columns): S0 | S1 | O0 | O1; the bf16 P of a tile overwrites the first half of its
@@ -97,6 +98,23 @@ __device__ __forceinline__ int lower_bound_pos(const int32_t* pos, int lo, int h
     if (int64_t(pos[mid]) < bound) lo = mid + 1; else hi = mid;
   }
   return lo;
+}
+// The same search by a whole warp: 32 probes per round instead of one, so a range of 2^17 rows
+// takes four dependent loads instead of seventeen.  Every lane returns the result.
+__device__ __forceinline__ int lower_bound_pos_warp(const int32_t* pos, int lo, int hi, int64_t bound, int lane) {
+  while (hi - lo > 32) {
+    const int step = (hi - lo + 32) / 33;                     // 32 probes cut the range into 33 pieces
+    const int idx = min(lo + (lane + 1) * step - 1, hi - 1);
+    const unsigned below = __ballot_sync(0xffffffffu, int64_t(pos[idx]) < bound);   // monotone: a prefix of ones
+    const int n = __popc(below);
+    const int new_lo = (n == 0) ? lo : min(lo + n * step, hi);   // probe n-1 was below the bound: so is everything up to it
+    const int new_hi = (n == 32) ? hi : min(lo + (n + 1) * step - 1, hi - 1);   // probe n was not: the answer is at or before it
+    lo = new_lo;
+    hi = max(new_hi, new_lo);
+  }
+  const int idx = lo + lane;
+  const unsigned below = __ballot_sync(0xffffffffu, idx < hi && int64_t(pos[idx]) < bound);
+  return lo + __popc(below);
 }
 
 template <int D>
@@ -199,19 +217,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     ptx::reg_dealloc<kRegsLean>();
     if (*abort_flag) {
       // a status word that was already set: do nothing
-    } else if (warp == 0) {
-      if (lane == 1) {
-        // ------------------------------------------------------------- geometry of the global range
-        pdl_wait();
-        const int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
-        const int64_t seg = st[TCA_ST_SEG_START];
-        const int n_global = int(st[TCA_ST_N_GLOBAL]);
-        const int vis_lo = lower_bound_pos(pos + seg, 0, n_global, c_lo);
+    } else if (warp == 2) {
+      // ------------------------------------------------------------- geometry of the global range
+      pdl_wait();
+      const int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
+      const int64_t seg = st[TCA_ST_SEG_START];
+      const int n_global = int(st[TCA_ST_N_GLOBAL]);
+      const int vis_lo = lower_bound_pos_warp(pos + seg, 0, n_global, c_lo, lane);
+      const int vis_hi = lower_bound_pos_warp(pos + seg, vis_lo, n_global, c_hi, lane);
+      if (lane == 0) {
         s_geo[0] = vis_lo;
-        s_geo[1] = lower_bound_pos(pos + seg, vis_lo, n_global, c_hi);
+        s_geo[1] = vis_hi;
         __threadfence_block();
         ptx::mbar_arrive(&bars[BAR_GEO]);
-      } else if (lane == 0) {
+      }
+    } else if (warp == 0) {
+      if (lane == 0) {
         // ------------------------------------------------------------- TMA producer
         ptx::mbar_arrive_expect_tx(&bars[BAR_Q], uint32_t(nh * Cfg::kQ));
         for (int h = 0; h < nh; ++h)
@@ -332,6 +353,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int row = quarter * 32 + lane;
         const int64_t i = i0 + row;
         const int64_t c_i = min(max(int64_t(0), i - window + 1), mb);
+        const int dc = int(c_i - c_lo), di = int(i - c_lo);   // window start and own position relative to the band
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
         const uint32_t s_addr = lane_addr + Cfg::colS(h);
         float m_run = -INFINITY, m_used = -INFINITY, l = 0.f;
@@ -353,11 +375,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             lo = 0;
             hi = nvis_i - 1 - geo.index(t) * BN;
           } else {
-            const int64_t p0 = geo.first(t);
-            lo = int(max(int64_t(-1), c_i - p0));
-            hi = int(min(int64_t(BN), i - p0));
+            const int off = geo.index(t) * BN;             // tile start relative to the band's first position
+            lo = max(-1, dc - off);
+            hi = min(BN, di - off);
           }
-          const bool masked = __any_sync(0xffffffffu, lo > 0 || hi < BN - 1);
+          // Per lane, no vote: the branch it guards only rewrites registers, so lanes may diverge in
+          // the few tiles that straddle a bound.
+          const bool masked = lo > 0 || hi < BN - 1;
           ok = __all_sync(0xffffffffu, ptx::mbar_wait(&bars[BAR_S + h], uint32_t(t) & 1u, abort_flag));   // uniform: the warp leaves together
           if (!ok) break;
           ptx::tc_fence_after();

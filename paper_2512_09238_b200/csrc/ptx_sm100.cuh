@@ -65,6 +65,34 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+// The same wait by polling without letting the hardware suspend the thread: lower wake-up latency
+// for a waiter that sits on the critical path, at the price of issue slots while it polls.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               uint64_t limit_ns = kWaitLimitNs) {
+  if (mbar_test_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 0;; ++i) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > limit_ns) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
 // What a tensor-core kernel does once its CTA has met again after an aborted wait: raise the
 // status word the host reads, then give bulk copies that were already issued time to land before
 // the shared memory they target is handed back.  (TMEM is freed by the caller, as on the normal
