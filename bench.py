@@ -100,7 +100,7 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.03)
         self.proc.terminate()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
@@ -111,22 +111,27 @@ class ClockSampler:
                 mx.append(float(parts[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(parts[2]))
+            except ValueError:
+                pass
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         busy = [x for x in sm if x > 0]
         return {"sm_mhz": float(np.median(busy)) if busy else None,
-                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm),
+                "power_w": float(np.median(pw)) if pw else None}
 
 
 # ----------------------------------------------------------------------------- workload on the device
 class Pipeline:
-    def __init__(self, wl, data, p, torch, B, host_io: bool = False):
+    def __init__(self, wl, data, p, torch, B, host_io: bool = False, flags: int = 0):
         self.wl, self.torch, self.B = wl, torch, B
         self.L, self.steps_decode = wl.L, wl.decode_steps
         T = wl.L + wl.decode_steps
         self.prm = B.make_params(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.block, wl.window,
-                                 alpha=wl.alpha, dtype=B.TCA_BF16 if wl.dtype == "bf16" else B.TCA_F32)
+                                 alpha=wl.alpha, dtype=B.TCA_BF16 if wl.dtype == "bf16" else B.TCA_F32, flags=flags)
         tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
 
         def host(a):
@@ -412,6 +417,10 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the 100 %-budget comparison run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="config5: skip the five-budget sweep")
+    ap.add_argument("--prefill-order", default="global", choices=["global", "band"],
+                    help="key-tile order of the prefill in the timed run: selected keys first, or the window band first "
+                         "(the band needs no selection, so the prefill then starts under score/select/compact)")
+    ap.add_argument("--no-order-compare", action="store_true", help="skip timing the other prefill order")
     ap.add_argument("--no-calibration", action="store_true", help="skip the offline calibration (Algorithm 1) leg")
     args = ap.parse_args()
 
@@ -472,7 +481,8 @@ def main():
     wl_rank = replica_workload(wl, rank)
     data = I.generate(wl_rank)
     p = I.budget_table(wl)
-    pipe = Pipeline(wl_rank, data, p, torch, B, host_io=not args.no_e2e)
+    order_flag = B.TCA_FLAG_PREFILL_BAND_FIRST if args.prefill_order == "band" else 0
+    pipe = Pipeline(wl_rank, data, p, torch, B, host_io=not args.no_e2e, flags=order_flag)
     peaks, peak_kind = load_peaks()
 
     def barrier():
@@ -516,7 +526,14 @@ def main():
            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": config,
            "ms_per_step_median": stages["step_median"], "ms_per_step_min": stages["step_min"],
            "decode_us_per_step": decode_us, "prefill_ms": prefill_ms, "clocks": clocks,
-           "gpu_launches": pipe.launches_per_step * args.steps}
+           "gpu_launches": pipe.launches_per_step * args.steps,
+           "prefill_order": args.prefill_order + " first"}
+    if clocks.get("power_w") and clocks.get("sm_mhz"):
+        # the prefill runs at the board's power cap: what limits it shows as energy per flop and as clocks per
+        # step (time x clock), not as time alone
+        out["energy"] = {"median_power_w": clocks["power_w"], "joule_per_step": clocks["power_w"] * ms_step * 1e-3,
+                         "prefill_ms_x_sm_mhz": stages["prefill"] * clocks["sm_mhz"],
+                         "note": "median board power and SM clock sampled during the timed steps"}
 
     tf_peak = peaks["bf16_tflops_sustained"]
     achieved_tf = work["prefill_flops"] / (stages["prefill"] * 1e-3) / 1e12
@@ -541,6 +558,21 @@ def main():
         "retained_fraction": work["retained_fraction"],
         "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
     }
+
+    if "energy" in out:
+        out["energy"]["picojoule_per_prefill_flop"] = (clocks["power_w"] * stages["prefill"] * 1e-3 /
+                                                       work["prefill_flops"] * 1e12)
+
+    if not args.no_order_compare and wl.dtype == "bf16":
+        # the same steps with the other key-tile order of the prefill (latency hiding: band first lets the prefill
+        # start under score/select/compact); both orders are parity-tested, the timed run uses --prefill-order
+        pipe.prm.flags ^= B.TCA_FLAG_PREFILL_BAND_FIRST
+        _, st_o, _ = timed(host_io=False)
+        pipe.prm.flags ^= B.TCA_FLAG_PREFILL_BAND_FIRST
+        other_ms = st_o["score_select"] + st_o["compact"] + st_o["prefill"]
+        names = ("band_first", "global_first") if args.prefill_order == "global" else ("global_first", "band_first")
+        out["prefill_order_compare"] = {names[0] + "_prefill_ms": other_ms, names[1] + "_prefill_ms": prefill_ms,
+                                        "stages_other_order": {k: st_o[k] for k in ("score_select", "compact", "prefill")}}
 
     if not args.no_dense:
         # this library's own dense path: the same calls with a 100 % budget (p_b = 1 for every head)

@@ -18,6 +18,11 @@ compact_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, int64_t
                int64_t* __restrict__ state) {
   const int u = blockIdx.y;
   int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
+  // Programmatic dependent launch: the prefill that follows may be scheduled now and, in its
+  // band-first order, work on the window band while this gather runs; this grid waits for the
+  // selection before it reads the index set.
+  pdl_launch_dependents();
+  pdl_wait();
   const int64_t seg = st[TCA_ST_SEG_START];
   const int64_t gcap = st[TCA_ST_GLOBAL_CAP];
   const int64_t off = offsets[u];
@@ -108,10 +113,9 @@ extern "C" int tca_compact_kv(const tca_params* prm, const void* K, const void* 
   const int pieces_per_row = int(prm->head_dim * elt_size(prm->dtype) / 16);
   if (max_rows == 0) max_rows = 1;  // still updates the device state
   dim3 grid(unsigned((max_rows + kRowsPerCta - 1) / kRowsPerCta), unsigned(U));
-  compact_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint4*>(K), static_cast<const uint4*>(V), L, pieces_per_row, tail_begin, idx,
-      offsets_dev, static_cast<uint4*>(c->k), static_cast<uint4*>(c->v), c->pos, c->state);
-  st = check_launch();
+  st = launch_pdl(compact_kernel, grid, dim3(kThreads), size_t(0), static_cast<cudaStream_t>(stream),
+                  static_cast<const uint4*>(K), static_cast<const uint4*>(V), L, pieces_per_row, tail_begin, idx,
+                  offsets_dev, static_cast<uint4*>(c->k), static_cast<uint4*>(c->v), c->pos, c->state);
   if (st != TCA_OK) return st;
   for (int64_t u = 0; u < U; ++u) {
     c->n_global[u] = offsets_host[u + 1] - offsets_host[u];

@@ -66,6 +66,11 @@ score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64
   const int u = blockIdx.y, chunk = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int grp = lane >> 2, j = lane & 3;
+  // Launched with programmatic dependent launch: the next kernel of the stream may be scheduled
+  // now (it waits for this grid itself), and this grid waits for its predecessor before it
+  // touches anything the predecessor may still be writing.
+  pdl_launch_dependents();
+  pdl_wait();
 
   __shared__ __align__(16) double qs[G][kChunks][QS];
   __shared__ double red_m[kWarps][G], red_l[kWarps][G];
@@ -191,6 +196,8 @@ score_finalize_kernel(const double* __restrict__ logits, const double* __restric
                       int64_t L, double* __restrict__ logscore, MetricOut mo) {
   const int u = blockIdx.y;
   const int tid = threadIdx.x;
+  pdl_launch_dependents();   // see score_logits_kernel
+  pdl_wait();
   __shared__ double lse[G];
   __shared__ double ls_s[kFinalizeRows];   // this CTA's log-scores, for the fused block metric
   // log-sum-exp of every head of the group from the per-chunk partials (warp g does head g)
@@ -257,15 +264,14 @@ int launch_score(const tca_params* prm, const void* q_last, const void* K, int64
                  const ScoreWs& ws, const MetricOut& mo, cudaStream_t stream) {
   const int U = prm->batch * prm->n_kv_heads;
   dim3 grid1(unsigned(ws.n_chunks), unsigned(U));
-  score_logits_kernel<T, D, G><<<grid1, kLogitThreads, 0, stream>>>(
-      static_cast<const T*>(q_last), static_cast<const T*>(K), L, double(prm->sm_scale), ws.logits,
-      ws.partials, int(ws.n_chunks));
-  int st = check_launch();
+  int st = launch_pdl(score_logits_kernel<T, D, G>, grid1, dim3(kLogitThreads), size_t(0), stream,
+                      static_cast<const T*>(q_last), static_cast<const T*>(K), L, double(prm->sm_scale), ws.logits,
+                      ws.partials, int(ws.n_chunks));
   if (st != TCA_OK) return st;
   dim3 grid2(unsigned((L + kFinalizeRows - 1) / kFinalizeRows), unsigned(U));
-  score_finalize_kernel<G><<<grid2, kThreads, 0, stream>>>(ws.logits, ws.partials, int(ws.n_chunks), L,
-                                                           logscore, mo);
-  return check_launch();
+  return launch_pdl(score_finalize_kernel<G>, grid2, dim3(kThreads), size_t(0), stream,
+                    static_cast<const double*>(ws.logits), static_cast<const double*>(ws.partials), int(ws.n_chunks), L,
+                    logscore, mo);
 }
 
 template <typename T, int D>

@@ -36,6 +36,8 @@ block_metric_kernel(const double* __restrict__ logscore, int64_t L, int m, int b
   const int u = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = blockIdx.x * kWarpsPerCta + warp;
+  pdl_launch_dependents();   // programmatic dependent launch: see score_logits_kernel
+  pdl_wait();
   if (j >= m) return;
   double h;
   if (mode == kMetricRandom) h = random_block_key(seed, u, j);
@@ -55,6 +57,8 @@ block_rank_kernel(const unsigned long long* __restrict__ hkey, int m, int n_kv_h
                   BudgetCounts counts, int32_t* __restrict__ t_ws, int32_t* __restrict__ t_out) {
   constexpr int kTile = 2048;
   __shared__ unsigned long long tile[kTile];
+  pdl_launch_dependents();
+  pdl_wait();
   const int u = blockIdx.y;
   const int part = threadIdx.x & (kRankParts - 1);
   const int j = blockIdx.x * kRankBlocks + (threadIdx.x >> 3);
@@ -92,6 +96,8 @@ block_topt_kernel(const double* __restrict__ logscore, int64_t L, int m, int b,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j0 = blockIdx.x * kWarpsPerCta;
   const int32_t* tu = t_ws + size_t(u) * m;
+  pdl_launch_dependents();
+  pdl_wait();
 
   // tokens kept by the blocks before this CTA's first block
   __shared__ int warp_sum[kWarpsPerCta];
@@ -162,6 +168,8 @@ flat_topb_kernel(const double* __restrict__ logscore, int64_t L, int64_t n_cand,
                  const int64_t* __restrict__ offsets, int32_t* __restrict__ idx) {
   const int u = blockIdx.x, tid = threadIdx.x;
   const double* ls = logscore + size_t(u) * L;
+  pdl_launch_dependents();
+  pdl_wait();
   const int64_t n_keep = offsets[u + 1] - offsets[u];
   if (n_keep <= 0) return;
   __shared__ unsigned hist[256];
@@ -235,24 +243,22 @@ int select_impl(const tca_params* prm, const double* logscore, int64_t L, const 
   if (m == 0) return TCA_OK;
   TCA_CHECK_ARG(idx != nullptr || !any);
   if (prm->flags & TCA_FLAG_FLAT_TOPB) {
-    flat_topb_kernel<<<unsigned(U), kFlatThreads, 0, s>>>(logscore, L, m * prm->block, offsets_dev, idx);
-    return check_launch();
+    return launch_pdl(flat_topb_kernel, dim3(unsigned(U)), dim3(kFlatThreads), size_t(0), s, logscore, L,
+                      m * prm->block, offsets_dev, idx);
   }
   int st;
   const unsigned gx = unsigned((m + kWarpsPerCta - 1) / kWarpsPerCta);
   if (!metric_done) {
-    block_metric_kernel<<<dim3(gx, unsigned(U)), kWarpsPerCta * 32, 0, s>>>(
-        logscore, L, int(m), prm->block, double(prm->alpha), metric_mode(prm), prm->seed, lay.hkey, h_out);
-    st = check_launch();
+    st = launch_pdl(block_metric_kernel, dim3(gx, unsigned(U)), dim3(kWarpsPerCta * 32), size_t(0), s, logscore, L,
+                    int(m), prm->block, double(prm->alpha), metric_mode(prm), prm->seed, lay.hkey, h_out);
     if (st != TCA_OK) return st;
   }
-  block_rank_kernel<<<dim3(unsigned((m + kRankBlocks - 1) / kRankBlocks), unsigned(U)), kRankThreads, 0, s>>>(
-      lay.hkey, int(m), prm->n_kv_heads, nK, counts, lay.t, t_out);
-  st = check_launch();
+  st = launch_pdl(block_rank_kernel, dim3(unsigned((m + kRankBlocks - 1) / kRankBlocks), unsigned(U)),
+                  dim3(kRankThreads), size_t(0), s, static_cast<const unsigned long long*>(lay.hkey), int(m),
+                  prm->n_kv_heads, nK, counts, lay.t, t_out);
   if (st != TCA_OK) return st;
-  block_topt_kernel<<<dim3(gx, unsigned(U)), kWarpsPerCta * 32, 0, s>>>(logscore, L, int(m), prm->block, lay.t,
-                                                                         offsets_dev, idx, lay.status);
-  return check_launch();
+  return launch_pdl(block_topt_kernel, dim3(gx, unsigned(U)), dim3(kWarpsPerCta * 32), size_t(0), s, logscore, L,
+                    int(m), prm->block, static_cast<const int32_t*>(lay.t), offsets_dev, idx, lay.status);
 }
 
 int check_select_args(const tca_params* prm, const double* logscore, int64_t L, const int32_t* n_k, int32_t nK,

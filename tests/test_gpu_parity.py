@@ -163,6 +163,70 @@ def test_prefill_by_row_ranges_is_bit_identical(runs, name):
 
 
 @pytest.mark.parametrize("name", ["bf16_gqa4", "bf16_d64_g2", "bf16_g7"])
+def test_band_first_order_matches_the_oracle_and_row_ranges(runs, name):
+    """TCA_FLAG_PREFILL_BAND_FIRST walks the window band before the selected keys (the order that
+    lets the prefill start before the selection has finished): every row against the oracle, and
+    row-range calls under the flag bit-identical to the single call under the flag."""
+    wl, data, p, run, oracle = runs(name)
+    run.prm.flags = B.TCA_FLAG_PREFILL_BAND_FIRST
+    try:
+        whole = H.gpu_prefill(run)
+        L = run.L
+        out = torch.full_like(run.dev["q"], float("nan"))
+        for (r0, r1) in [(384, L), (0, 128), (128, 384)]:
+            ws = B.alloc_workspace(run.prm, L, B.TCA_OP_PREFILL)
+            B.tca_attn_prefill_rows(run.prm, run.dev["q"], run.dev["k"], run.dev["v"], L, r0, r1, run.cache, out, ws)
+            assert B.tca_ws_status(ws) == B.TCA_OK
+        assert torch.equal(whole.view(torch.uint8), out.view(torch.uint8))
+    finally:
+        run.prm.flags = 0
+    got = H.from_device(whole)
+    scale, G = H.scale_of(wl), wl.group
+    for s_ in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            T = _oracle_T(run, wl, s_ * wl.n_kv_heads + h)
+            K, V = I.widen(data["k"][s_, h, :wl.L]), I.widen(data["v"][s_, h, :wl.L])
+            for g in range(G):
+                want = O.attention_rows(I.widen(data["q"][s_, h * G + g, :wl.L]), K, V, T, wl.window, scale)
+                H.check_attention(got[s_, h * G + g], want, wl.dtype, f"{name} band first head {h * G + g}")
+
+
+@pytest.mark.parametrize("order", [0, B.TCA_FLAG_PREFILL_BAND_FIRST])
+def test_the_chain_without_host_synchronisation_equals_the_synchronised_one(order):
+    """score+select, compact and prefill are launched with programmatic dependent launch: each may
+    be scheduled while its predecessor is still running and waits for it on the device.  Enqueued
+    back to back, several times over the same buffers and with a changing input, the results must be
+    those of running every call to completion first."""
+    wl = SMALL["bf16_gqa4"].scaled(L=1400, seed=61)
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    ref = H.gpu_select_compact(wl, data, p, flags=order)           # synchronises between the stages
+    want = H.gpu_prefill(ref)
+    torch.cuda.synchronize()
+    prm, L = ref.prm, wl.L
+    U = wl.batch * wl.n_kv_heads
+    offsets_dev = torch.from_numpy(ref.offsets).cuda()
+    q_last = ref.dev["q"][:, :, L - 1, :].contiguous()
+    other = (ref.dev["k"].float() * 0.5).to(torch.bfloat16)        # a different K: different selection, different cache
+    logscore = torch.empty(U, L, dtype=torch.float64, device="cuda")
+    idx = torch.empty_like(ref.idx)
+    ws_ss = B.alloc_workspace(prm, L, B.TCA_OP_SCORE_SELECT)
+    ws_pf = B.alloc_workspace(prm, L, B.TCA_OP_PREFILL)
+    tk = np.tile(ref.tbar, wl.batch).astype(np.int64)
+    cache = B.Cache(prm, np.tile(ref.n_sel, wl.batch), wl.window + wl.block, tk)
+    out = torch.empty_like(ref.dev["q"])
+    for K_dev in (other, ref.dev["k"], other, ref.dev["k"]):       # ends on the reference input
+        B.tca_score_select(prm, q_last, K_dev, L, ref.n_k, logscore, idx, offsets_dev, None, None, ws_ss)
+        B.tca_compact_kv(prm, K_dev, ref.dev["v"], L, idx, offsets_dev, ref.offsets, cache)
+        B.tca_attn_prefill(prm, ref.dev["q"], K_dev, ref.dev["v"], L, cache, out, ws_pf)
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(ws_pf) == B.TCA_OK
+    assert torch.equal(idx, ref.idx)
+    assert torch.equal(cache.pos, ref.cache.pos) and torch.equal(cache.k.view(torch.int16), ref.cache.k.view(torch.int16))
+    assert torch.equal(out.view(torch.uint8), want.view(torch.uint8))
+
+
+@pytest.mark.parametrize("name", ["bf16_gqa4", "bf16_d64_g2", "bf16_g7"])
 def test_bf16_prefill_reference_kernel_agrees(runs, name):
     """The FP32-pipe kernel and the default bf16 kernel see the same inputs."""
     wl, data, p, run, oracle = runs(name)
@@ -262,6 +326,9 @@ def test_degenerate_lengths_on_the_tensor_core_paths(L, w, b, d, G):
     p = I.budget_table(wl)
     run = H.gpu_select_compact(wl, data, p)
     out = H.from_device(H.gpu_prefill(run))
+    run.prm.flags = B.TCA_FLAG_PREFILL_BAND_FIRST
+    out_band = H.from_device(H.gpu_prefill(run))
+    run.prm.flags = 0
     dec = H.from_device(H.gpu_decode(run, run.dev["q"][:, :, L - 1, :].contiguous()))
     scale = H.scale_of(wl)
     for h in range(2):
@@ -274,6 +341,7 @@ def test_degenerate_lengths_on_the_tensor_core_paths(L, w, b, d, G):
             Q = I.widen(data["q"][0, h * G + g])
             want = O.attention_rows(Q, K, V, res["T"], w, scale)
             H.check_attention(out[0, h * G + g], want, "bf16", f"prefill L={L} w={w} b={b} d={d}")
+            H.check_attention(out_band[0, h * G + g], want, "bf16", f"prefill, band first, L={L} w={w} b={b} d={d}")
             want_dec = O.attention_over_set(Q[L - 1], K[res["T"]], V[res["T"]], scale)
             H.check_attention(dec[0, h * G + g], want_dec, "bf16", f"decode L={L} w={w} b={b} d={d}")
 
