@@ -34,7 +34,7 @@ def _check_selection(wl, data, p, pipe, units):
         t = np.bincount(S // wl.block, minlength=res["m"])
         accepted += H.compare_selection(res, S, t, wl.block)
         sel[u] = S
-    assert accepted <= 4
+    assert accepted <= max(4, len(list(units)) // 4)      # differences inside the 1e-5 band stay rare
     return sel
 
 
@@ -66,6 +66,21 @@ def test_config3_prefill_32k():
     # retained-token counts equal each head's budget
     for u in range(pipe.U):
         assert len(sel[u]) == pipe.n_sel[u % wl.n_kv_heads] == pipe.cache.n_global[u]
+
+
+def test_config3_prefill_32k_band_first():
+    """The same configuration with the window band walked first (TCA_FLAG_PREFILL_BAND_FIRST), the
+    whole chain enqueued without host synchronisation: sampled rows of every unit against the oracle."""
+    wl = I.WORKLOADS["config3"]
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    pipe = bench.Pipeline(wl, data, p, torch, B, host_io=False, flags=B.TCA_FLAG_PREFILL_BAND_FIRST)
+    pipe.step()
+    pipe.step()
+    torch.cuda.synchronize()
+    assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    sel = _check_selection(wl, data, p, pipe, range(pipe.U))
+    _check_prefill_rows(wl, data, pipe, sel, n_random=6)
 
 
 def test_config4_prefill_128k_then_256_decode_steps():
@@ -125,8 +140,8 @@ def test_config2_decode_32k_batch4_and_dense_decode():
     out = torch.empty_like(pipe.q_last)
     B.tca_attn_decode(pipe.prm, pipe.q_last, pipe.cache, out, pipe.ws_decode)
     torch.cuda.synchronize()
-    units = [0, 7, 13, 22, 31]
-    sel = _check_selection(wl, data, p, pipe, units)
+    sel = _check_selection(wl, data, p, pipe, range(pipe.U))       # the selection of every unit
+    units = [0, 7, 13, 22, 31]                                      # decode outputs of five of them
     got = H.from_device(out)
     scale = H.scale_of(wl)
     for u in units:
@@ -166,10 +181,10 @@ def test_config5_budget_sweep_64k(frac):
     pipe.step()
     torch.cuda.synchronize()
     assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    sel = _check_selection(wl, data, p, pipe, range(pipe.U))       # the selection of every unit
     units = [0, 5, 11, 15]
-    sel = _check_selection(wl, data, p, pipe, units)
     m = wl.n_blocks
-    for u in units:   # uniform budget: every head keeps the same count, and sees it in its cache
+    for u in range(pipe.U):   # uniform budget: every head keeps the same count, and sees it in its cache
         assert len(sel[u]) == pipe.n_sel[0]
         assert abs(len(sel[u]) / (m * wl.block) - frac) < 0.01
     _check_prefill_rows(wl, data, pipe, {u: sel[u] for u in units[:2]}, n_random=4)
