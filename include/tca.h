@@ -258,6 +258,26 @@ int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, c
                           void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same attention (Eq. 2) without a cache: the selected keys are fetched from K and V
+ * themselves, by index, inside the attention kernel (Appendix C, "Memory Access Optimization":
+ * gathering fused into the consumer instead of a separate compaction pass).  For a caller that
+ * only prefills, or that builds the decode cache later: no tca_compact_kv, no cache memory.
+ * O is bit-identical to tca_compact_kv + tca_attn_prefill_rows over the same selection.
+ *   idx, offsets_dev  DEVICE, as written by / given to tca_select: unit u's selected positions
+ *                     are idx[offsets_dev[u] .. offsets_dev[u+1]), ascending; not modified
+ *   row_begin, row_end  as in tca_attn_prefill_rows ([0, L) for the whole prefill)
+ *   ws                as in tca_attn_prefill (sticky status word in word 0)
+ * bf16 only, on the tensor-core kernel (TCA_ERR_UNSUPPORTED for TCA_F32 or
+ * TCA_FLAG_PREFILL_SIMT, and when batch * n_kv_heads * L >= 2^31: the row coordinates of a
+ * gather are 32-bit).  TCA_FLAG_PREFILL_BAND_FIRST applies.  The index set is trusted to hold
+ * candidate positions (< m*b); the range-checked build verifies it (TCA_ERR_BOUNDS in ws).
+ */
+int tca_attn_prefill_gather(const tca_params* prm, const void* Q, const void* K, const void* V,
+                            int64_t L, int64_t row_begin, int64_t row_end,
+                            const int32_t* idx, const int64_t* offsets_dev, void* O,
+                            void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Offline calibration, Algorithm 1 and Eq. 4 (Section 4.1, "Cumulative-Score Configuration
  * Determination").  It produces the per-head configuration p* that the functions above take
  * as an input.  Three calls:

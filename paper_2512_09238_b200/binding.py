@@ -35,7 +35,7 @@ EXPORTS = (
     "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
     "tca_calib_colmean", "tca_calib_score", "tca_calib_choose", "tca_calib_candidates",
     "tca_decode_static_status", "tca_selftest_wait_expiry", "tca_score_select", "tca_build_info",
-    "tca_cache_status",
+    "tca_cache_status", "tca_attn_prefill_gather",
 )
 
 
@@ -86,6 +86,7 @@ def load_library(path: str) -> C.CDLL:
     L.tca_compact_kv.argtypes = [P, vp, vp, i64, vp, vp, vp, D, vp]
     L.tca_attn_prefill.argtypes = [P, vp, vp, vp, i64, D, vp, vp, sz, vp]
     L.tca_attn_prefill_rows.argtypes = [P, vp, vp, vp, i64, i64, i64, D, vp, vp, sz, vp]
+    L.tca_attn_prefill_gather.argtypes = [P, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]
     L.tca_calib_colmean.argtypes = [P, vp, vp, i64, vp, vp, sz, vp]
     L.tca_calib_score.argtypes = [P, vp, i64, vp, vp, vp, vp]
     L.tca_calib_choose.argtypes = [vp, vp, C.c_int, C.c_double]
@@ -233,6 +234,12 @@ def tca_attn_prefill_rows(prm, Q, K, V, L, row_begin, row_end, cache: "Cache", O
     _check(lib().tca_attn_prefill_rows(C.byref(prm), _dev(Q), _dev(K), _dev(V), L, row_begin, row_end,
                                        C.byref(cache.desc), _dev(O), *_ws_args(ws), _stream(stream)),
            "tca_attn_prefill_rows")
+
+
+def tca_attn_prefill_gather(prm, Q, K, V, L, row_begin, row_end, idx, offsets_dev, O, ws, stream=None) -> None:
+    _check(lib().tca_attn_prefill_gather(C.byref(prm), _dev(Q), _dev(K), _dev(V), L, row_begin, row_end,
+                                         _dev(idx), _dev(offsets_dev), _dev(O), *_ws_args(ws), _stream(stream)),
+           "tca_attn_prefill_gather")
 
 
 def tca_attn_decode(prm, q, cache: "Cache", O, ws, stream=None) -> None:

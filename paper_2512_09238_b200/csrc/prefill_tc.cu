@@ -117,7 +117,11 @@ __device__ __forceinline__ int lower_bound_pos_warp(const int32_t* pos, int lo, 
   return lo + __popc(below);
 }
 
-template <int D>
+// kGather: the selected keys are not read from a compacted cache but fetched from K and V
+// themselves, row by row, by the producer (tile::gather4); `pos` is then the index set that the
+// selection wrote, `state` its per-unit offsets, and map_ck / map_cv are row-gather maps over the
+// flattened K and V.
+template <int D, bool kGather>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_ck,
@@ -202,7 +206,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (!ptx::mbar_wait(&bars[BAR_GEO], 0, abort_flag)) return false;
     pdl_wait();                                   // the cache rows read from here on are visible to this thread
     const int n_gt = (s_geo[1] + BN - 1) / BN;
-    geo.seg = state[size_t(u) * TCA_STATE_WORDS + TCA_ST_SEG_START];
+    geo.seg = kGather ? state[u] : state[size_t(u) * TCA_STATE_WORDS + TCA_ST_SEG_START];
     if (geo.band_first) geo.n_b = n_gt; else geo.n_a = n_gt;
     geo_known = true;
     return true;
@@ -221,8 +225,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       // ------------------------------------------------------------- geometry of the global range
       pdl_wait();
       const int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
-      const int64_t seg = st[TCA_ST_SEG_START];
-      const int n_global = int(st[TCA_ST_N_GLOBAL]);
+      const int64_t seg = kGather ? state[u] : st[TCA_ST_SEG_START];
+      const int n_global = kGather ? int(state[u + 1] - state[u]) : int(st[TCA_ST_N_GLOBAL]);
       const int vis_lo = lower_bound_pos_warp(pos + seg, 0, n_global, c_lo, lane);
       const int vis_hi = lower_bound_pos_warp(pos + seg, vis_lo, n_global, c_hi, lane);
       if (lane == 0) {
@@ -232,44 +236,80 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         ptx::mbar_arrive(&bars[BAR_GEO]);
       }
     } else if (warp == 0) {
-      if (lane == 0) {
-        // ------------------------------------------------------------- TMA producer
-        ptx::mbar_arrive_expect_tx(&bars[BAR_Q], uint32_t(nh * Cfg::kQ));
-        for (int h = 0; h < nh; ++h)
-          for (int half = 0; half < Cfg::NH; ++half)
-            ptx::tma_load_3d(smem + Cfg::offQ + h * Cfg::kQ + half * kHalfBytes, &map_q, half * 64, int(i0),
-                             hq0 + h, &bars[BAR_Q]);
-        bool ok = band_first || learn_geometry();
+      // ------------------------------------------------------------- TMA producer
+      // One lane issues the box loads.  Row gathers are issued by the whole warp, a lane for every
+      // four rows of the tile, so there all lanes walk the loop and every wait is made warp-uniform.
+      if (kGather || lane == 0) {
+        auto pwait = [&](uint64_t* bar, uint32_t parity) -> bool {
+          const bool r = ptx::mbar_wait(bar, parity, abort_flag);
+          if constexpr (kGather) return __all_sync(0xffffffffu, r); else return r;
+        };
+        auto plearn = [&]() -> bool {
+          if constexpr (kGather) return learn_geometry_warp(); else return learn_geometry();
+        };
+        if (lane == 0) {
+          ptx::mbar_arrive_expect_tx(&bars[BAR_Q], uint32_t(nh * Cfg::kQ));
+          for (int h = 0; h < nh; ++h)
+            for (int half = 0; half < Cfg::NH; ++half)
+              ptx::tma_load_3d(smem + Cfg::offQ + h * Cfg::kQ + half * kHalfBytes, &map_q, half * 64, int(i0),
+                               hq0 + h, &bars[BAR_Q]);
+        }
+        bool ok = band_first || plearn();
         // load n: n = 0 is K of tile 0; n = 2t+1 is V of tile t; n = 2t+2 is K of tile t+1.  V_t and
         // K_t+1 share the barrier pair t % kPairs (the issuer needs them together).
         for (int n = 0; ok; ++n) {
           const int is_v = n & 1;
           const int t = is_v ? (n - 1) >> 1 : n >> 1;          // the tile this load belongs to
-          if (t >= geo.n_a && !geo_known) { ok = learn_geometry(); if (!ok) break; }
+          if (t >= geo.n_a && !geo_known) { ok = plearn(); if (!ok) break; }
           if (t >= geo.n_a + geo.n_b) {
             // past the last tile: the last pair holds V only, its barrier still expects two arrivals
-            if (!is_v && t > 0) ptx::mbar_arrive(&bars[BAR_FULL + (t - 1) % kPairs]);
+            if (!is_v && t > 0 && lane == 0) ptx::mbar_arrive(&bars[BAR_FULL + (t - 1) % kPairs]);
             break;
           }
           const int slot = n % kRing;
           if (n >= kRing) {                                    // the slot's previous tile must have been consumed
             const int r = n - kRing;
-            if (r == 0) ok = ptx::mbar_wait(&bars[BAR_K0_EMPTY], 0, abort_flag);
+            if (r == 0) ok = pwait(&bars[BAR_K0_EMPTY], 0);
             else {
               const int tr = (r - 1) >> 1;
-              ok = ptx::mbar_wait(&bars[BAR_EMPTY + tr % kPairs], uint32_t(tr / kPairs) & 1u, abort_flag);
+              ok = pwait(&bars[BAR_EMPTY + tr % kPairs], uint32_t(tr / kPairs) & 1u);
             }
             if (!ok) break;
           }
           uint64_t* full = (n == 0) ? &bars[BAR_K0_FULL] : &bars[BAR_FULL + ((n - 1) >> 1) % kPairs];
-          ptx::mbar_arrive_expect_tx(full, uint32_t(Cfg::kKV));
+          if (lane == 0) ptx::mbar_arrive_expect_tx(full, uint32_t(Cfg::kKV));
           uint8_t* dst = smem + Cfg::offKV + slot * Cfg::kKV;
-          const int y = int(geo.first(t));
-          for (int half = 0; half < Cfg::NH; ++half) {
-            if (geo.is_global(t))
-              ptx::tma_load_2d(dst + half * kHalfBytes, is_v ? &map_cv : &map_ck, half * 64, y, full);
-            else
-              ptx::tma_load_3d(dst + half * kHalfBytes, is_v ? &map_v : &map_k, half * 64, y, u, full);
+          if (kGather && geo.is_global(t)) {
+            // Rows 4*lane .. 4*lane+3 of the tile are the unit's selected keys number first + 4*lane ...
+            // A tile that reaches past the keys visible to this query tile repeats the last visible
+            // one: the mask gives those columns an exact zero weight, the row only has to be finite.
+            __syncwarp();                                      // the expectation is posted before any piece can land
+            const int32_t* sel = pos + geo.seg;
+            const int last = s_geo[1] - 1;                     // >= 0: there is at least one global tile
+            const int first = geo.index(t) * BN + 4 * lane;
+            int rows[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              int64_t p = sel[min(first + k, last)];
+              if constexpr (kDebugBounds) {
+                if (p < 0 || p >= mb) {                        // a selected index names a candidate token
+                  report_bounds_ws(status, kBoundsSelectedIndex, p);
+                  p = 0;
+                }
+              }
+              rows[k] = int(int64_t(u) * L + p);
+            }
+            for (int half = 0; half < Cfg::NH; ++half)
+              ptx::tma_gather4_2d(dst + half * kHalfBytes + lane * 512, is_v ? &map_cv : &map_ck, half * 64, rows[0],
+                                  rows[1], rows[2], rows[3], full);
+          } else if (lane == 0) {
+            const int y = int(geo.first(t));
+            for (int half = 0; half < Cfg::NH; ++half) {
+              if (geo.is_global(t))
+                ptx::tma_load_2d(dst + half * kHalfBytes, is_v ? &map_cv : &map_ck, half * 64, y, full);
+              else
+                ptx::tma_load_3d(dst + half * kHalfBytes, is_v ? &map_v : &map_k, half * 64, y, u, full);
+            }
           }
         }
       }
@@ -526,7 +566,9 @@ bool cached_map(CUtensorMap* out, const void* base, int D, int64_t rows, int64_t
   MapEntry& slot = g_maps[g_map_next];
   g_map_next = (g_map_next + 1) % 16;
   slot.key = MapKey{nullptr, 0, 0, 0};
-  if (!encode_map(&slot.map, base, D, rows, heads, rows)) return false;
+  const bool encoded = heads < 0 ? encode_gather_map(&slot.map, base, D, rows)   // heads = -1: a row-gather map
+                                 : encode_map(&slot.map, base, D, rows, heads, rows);
+  if (!encoded) return false;
   slot.key = key;
   *out = slot.map;
   return true;
@@ -536,21 +578,29 @@ bool cached_map(CUtensorMap* out, const void* base, int D, int64_t rows, int64_t
 
 size_t prefill_tc_ws_bytes(const tca_params*) { return 256; }   // the status word
 
-template <int D>
-int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
-                      int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O, void* ws,
-                      cudaStream_t stream) {
+// The selected keys come either from the cache (c != nullptr) or, by row gathers, from K and V
+// themselves (c == nullptr; idx and offsets_dev are what the selection wrote / was given).
+template <int D, bool kGather>
+int launch_prefill_tc_impl(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
+                           int64_t row_begin, int64_t row_end, const tca_cache_desc* c, const int32_t* idx,
+                           const int64_t* offsets_dev, void* O, void* ws, cudaStream_t stream) {
   using Cfg = TcCfg<D>;
   const int64_t U = int64_t(prm->batch) * prm->n_kv_heads;
   const int G = prm->n_q_heads / prm->n_kv_heads;
   CUtensorMap mq, mk, mv, mck, mcv;
-  // The cache maps cover the whole flattened cache (rows past the end read as zero); a tile that
-  // reaches past a unit's visible prefix reads other finite rows, which the mask turns into exact zeros.
   if (!cached_map(&mq, Q, D, L, int64_t(prm->batch) * prm->n_q_heads) || !cached_map(&mk, K, D, L, U) ||
-      !cached_map(&mv, V, D, L, U) || !cached_map(&mck, c->k, D, c->rows_total, 0) ||
-      !cached_map(&mcv, c->v, D, c->rows_total, 0))
+      !cached_map(&mv, V, D, L, U))
     return TCA_ERR_CUDA;
-  auto kern = prefill_tc_kernel<D>;
+  if constexpr (kGather) {
+    if (U * L >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;   // row coordinates are 32-bit
+    if (!cached_map(&mck, K, D, U * L, -1) || !cached_map(&mcv, V, D, U * L, -1)) return TCA_ERR_CUDA;
+  } else {
+    // The cache maps cover the whole flattened cache (rows past the end read as zero); a tile that
+    // reaches past a unit's visible prefix reads other finite rows, which the mask turns into exact zeros.
+    if (!cached_map(&mck, c->k, D, c->rows_total, 0) || !cached_map(&mcv, c->v, D, c->rows_total, 0))
+      return TCA_ERR_CUDA;
+  }
+  auto kern = prefill_tc_kernel<D, kGather>;
   TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::bytes));
   const int tile0 = int(row_begin / BM);
   const int n_qtiles = int((row_end - row_begin + BM - 1) / BM);
@@ -558,16 +608,36 @@ int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const
   const int64_t n_ctas = int64_t(n_qtiles) * U * pairs;
   if (n_ctas >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;
   const int64_t mb = num_blocks(prm, L) * prm->block;
-  return launch_pdl(kern, dim3(unsigned(n_ctas)), dim3(kThreads), size_t(Cfg::bytes), stream, mq, mk, mv, mck, mcv,
-                    static_cast<const int32_t*>(c->pos), static_cast<const int64_t*>(c->state), L, prm->n_q_heads,
-                    prm->n_kv_heads, prm->window, mb, prm->sm_scale * 1.4426950408889634f,
-                    static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws), n_qtiles, pairs, tile0,
-                    (prm->flags & TCA_FLAG_PREFILL_BAND_FIRST) ? 1 : 0);
+  const int32_t* pos = kGather ? idx : static_cast<const int32_t*>(c->pos);
+  const int64_t* state = kGather ? offsets_dev : static_cast<const int64_t*>(c->state);
+  return launch_pdl(kern, dim3(static_cast<unsigned>(n_ctas)), dim3(kThreads), size_t(Cfg::bytes), stream, mq, mk, mv,
+                    mck, mcv, pos, state, L, prm->n_q_heads, prm->n_kv_heads, prm->window, mb,
+                    prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws),
+                    n_qtiles, pairs, tile0, (prm->flags & TCA_FLAG_PREFILL_BAND_FIRST) ? 1 : 0);
+}
+
+template <int D>
+int launch_prefill_tc(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
+                      int64_t row_begin, int64_t row_end, const tca_cache_desc* c, void* O, void* ws,
+                      cudaStream_t stream) {
+  return launch_prefill_tc_impl<D, false>(prm, Q, K, V, L, row_begin, row_end, c, nullptr, nullptr, O, ws, stream);
+}
+template <int D>
+int launch_prefill_tc_gather(const tca_params* prm, const void* Q, const void* K, const void* V, int64_t L,
+                             int64_t row_begin, int64_t row_end, const int32_t* idx, const int64_t* offsets_dev,
+                             void* O, void* ws, cudaStream_t stream) {
+  return launch_prefill_tc_impl<D, true>(prm, Q, K, V, L, row_begin, row_end, nullptr, idx, offsets_dev, O, ws,
+                                         stream);
 }
 
 template int launch_prefill_tc<64>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
                                    int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
 template int launch_prefill_tc<128>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
                                     int64_t, const tca_cache_desc*, void*, void*, cudaStream_t);
+
+template int launch_prefill_tc_gather<64>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
+                                          int64_t, const int32_t*, const int64_t*, void*, void*, cudaStream_t);
+template int launch_prefill_tc_gather<128>(const tca_params*, const void*, const void*, const void*, int64_t, int64_t,
+                                           int64_t, const int32_t*, const int64_t*, void*, void*, cudaStream_t);
 
 }  // namespace tca
