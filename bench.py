@@ -213,6 +213,29 @@ class Pipeline:
             B.tca_attn_decode(prm, self.qd[s], self.cache, self.Od[s], self.ws_decode)
         if mark: self._ev("t_decode")
 
+    def time_gather_prefill(self, reps: int = 3):
+        """score + select, then the prefill that gathers the selected rows itself (no compaction, no cache):
+        the prefill-only form of the path, timed with CUDA events, median of `reps` after one warm-up."""
+        B, prm, L, torch = self.B, self.prm, self.L, self.torch
+        ms_sel, ms_pf = [], []
+        for r in range(reps + 1):
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record()
+            B.tca_score_select(prm, self.q_last, self.Kp, L, self.n_k, self.logscore, self.idx, self.offsets_dev, None,
+                               None, self.ws_score_select)
+            e[1].record()
+            B.tca_attn_prefill_gather(prm, self.Qp, self.Kp, self.Vp, L, 0, L, self.idx, self.offsets_dev, self.O,
+                                      self.ws_prefill)
+            e[2].record()
+            torch.cuda.synchronize()
+            if r > 0:
+                ms_sel.append(e[0].elapsed_time(e[1]))
+                ms_pf.append(e[1].elapsed_time(e[2]))
+        assert B.tca_ws_status(self.ws_prefill) == B.TCA_OK
+        sel, pf = float(np.median(ms_sel)), float(np.median(ms_pf))
+        return {"score_select_ms": sel, "prefill_ms": pf, "total_ms": sel + pf, "reps": reps,
+                "note": "tca_attn_prefill_gather: selected rows fetched from K, V by TMA row gathers in the producer"}
+
     def step_from_host(self, mark: bool = False):
         """The same step with every input in pinned host memory and every output read back.
 
@@ -573,6 +596,10 @@ def main():
         names = ("band_first", "global_first") if args.prefill_order == "global" else ("global_first", "band_first")
         out["prefill_order_compare"] = {names[0] + "_prefill_ms": other_ms, names[1] + "_prefill_ms": prefill_ms,
                                         "stages_other_order": {k: st_o[k] for k in ("score_select", "compact", "prefill")}}
+
+    if not args.no_order_compare and wl.dtype == "bf16":
+        out["prefill_gather"] = pipe.time_gather_prefill(reps=max(3, min(5, args.steps)))
+        out["prefill_gather"]["with_compaction_ms"] = prefill_ms
 
     if not args.no_dense:
         # this library's own dense path: the same calls with a 100 % budget (p_b = 1 for every head)

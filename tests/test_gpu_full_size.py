@@ -83,6 +83,24 @@ def test_config3_prefill_32k_band_first():
     _check_prefill_rows(wl, data, pipe, sel, n_random=6)
 
 
+@pytest.mark.parametrize("name", ["config3", "config4"])
+def test_gather_prefill_equals_the_cache_path_at_full_size(name):
+    """tca_attn_prefill_gather (selected rows fetched from K, V inside the attention kernel) over the
+    selection of the timed pipeline: every element of O bit for bit equal to compaction + prefill,
+    whose sampled rows the tests above compare with the oracle."""
+    wl = I.WORKLOADS[name]
+    data, p, pipe = _pipeline(wl)
+    pipe.steps_decode = 0
+    pipe.step()
+    torch.cuda.synchronize()
+    via_cache = pipe.O.clone()
+    pipe.O.fill_(float("nan"))
+    t = pipe.time_gather_prefill(reps=1)
+    assert t["prefill_ms"] > 0
+    assert B.tca_ws_status(pipe.ws_prefill) == B.TCA_OK
+    assert torch.equal(pipe.O.view(torch.uint8), via_cache.view(torch.uint8))
+
+
 def test_config4_prefill_128k_then_256_decode_steps():
     wl = I.WORKLOADS["config4"]
     data, p, pipe = _pipeline(wl)
