@@ -2,6 +2,7 @@
 // layouts, cache descriptor upload.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -30,6 +31,23 @@ int check_params(const tca_params* prm) {
   if (!is_pow2(prm->block) || prm->block > kMaxBlock) return TCA_ERR_UNSUPPORTED;
   if (prm->n_q_heads / prm->n_kv_heads > kMaxGroup) return TCA_ERR_UNSUPPORTED;
   return TCA_OK;
+}
+
+namespace {
+std::mutex g_device_mutex;
+int g_sm_count[kMaxDevices] = {};
+}  // namespace
+
+int sm_count() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (g_sm_count[dev] == 0) {
+    int n = 0;
+    g_sm_count[dev] =
+        (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+  }
+  return g_sm_count[dev];
 }
 
 ScoreWs score_ws_layout(const tca_params* prm, int64_t L, void* ws) {

@@ -61,6 +61,10 @@ inline size_t elt_size(int dtype) { return dtype == TCA_BF16 ? 2 : 4; }
 // ------------------------------------------------------------------ workspace layouts
 // score: logits [U][G][L] double, then partials [U][n_chunks][G][2] double.
 constexpr int kScoreChunkRows = 1024;  // rows of K per CTA of the logit kernel
+// Streaming multiprocessors of the current device, looked up once per device (api.cu).
+constexpr int kMaxDevices = 64;
+int sm_count();
+
 struct ScoreWs {
   double* logits;
   double* partials;

@@ -356,23 +356,6 @@ decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restri
   }
 }
 
-// Streaming multiprocessors of the current device, looked up once per device.
-constexpr int kMaxDevices = 64;
-std::mutex g_device_mutex;
-int g_sm_count[kMaxDevices] = {};
-
-inline int sm_count() {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
-  std::lock_guard<std::mutex> lock(g_device_mutex);
-  if (g_sm_count[dev] == 0) {
-    int n = 0;
-    g_sm_count[dev] =
-        (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
-  }
-  return g_sm_count[dev];
-}
-
 // Rows per CTA: enough CTAs for two per SM, at least one softmax round each.
 inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_sm, int64_t* max_len_out) {
   int64_t total = 0, max_len = 0;

@@ -36,10 +36,13 @@ __device__ __forceinline__ void merge_ml(double& m, double& l, double m2, double
 
 // 16-byte chunk -> doubles
 __device__ __forceinline__ void chunk_to_double(const uint4& w, double (&x)[8], __nv_bfloat16) {
-  x[0] = bf16_lo_to_double(w.x); x[1] = bf16_hi_to_double(w.x);
-  x[2] = bf16_lo_to_double(w.y); x[3] = bf16_hi_to_double(w.y);
-  x[4] = bf16_lo_to_double(w.z); x[5] = bf16_hi_to_double(w.z);
-  x[6] = bf16_lo_to_double(w.w); x[7] = bf16_hi_to_double(w.w);
+  // one shift or mask and one hardware conversion per element: the conversion unit runs beside the
+  // fp64 pipe, whereas placing the bits by integer arithmetic costs more issue slots than the
+  // multiply-adds that use the value
+  x[0] = double(bf16_lo(w.x)); x[1] = double(bf16_hi(w.x));
+  x[2] = double(bf16_lo(w.y)); x[3] = double(bf16_hi(w.y));
+  x[4] = double(bf16_lo(w.z)); x[5] = double(bf16_hi(w.z));
+  x[6] = double(bf16_lo(w.w)); x[7] = double(bf16_hi(w.w));
 }
 __device__ __forceinline__ void chunk_to_double(const uint4& w, double (&x)[8], float) {
   x[0] = double(__uint_as_float(w.x)); x[1] = double(__uint_as_float(w.y));
@@ -57,7 +60,7 @@ constexpr int kLogitThreads = 128;
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kLogitThreads)
 score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64_t L, double sm_scale,
-                    double* __restrict__ logits, double* __restrict__ partials, int n_chunks) {
+                    double* __restrict__ logits, double* __restrict__ partials, int n_chunks, int rows_per_cta) {
   constexpr int EPC = 16 / int(sizeof(T));          // elements per 16-byte chunk
   constexpr int kChunks = D / EPC;                  // chunks per row
   constexpr int kIters = kChunks / 4;               // chunks per lane
@@ -82,8 +85,8 @@ score_logits_kernel(const T* __restrict__ q_last, const T* __restrict__ K, int64
 
   const T* Ku = K + size_t(u) * L * D;
   double* logits_u = logits + size_t(u) * G * L;
-  const int64_t row0 = int64_t(chunk) * kScoreChunkRows;
-  const int64_t row_end = min(row0 + int64_t(kScoreChunkRows), L);
+  const int64_t row0 = int64_t(chunk) * rows_per_cta;
+  const int64_t row_end = min(row0 + int64_t(rows_per_cta), L);
   double run_m[G], run_l[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) { run_m[g] = 0.0; run_l[g] = 0.0; }
@@ -200,7 +203,20 @@ score_finalize_kernel(const double* __restrict__ logits, const double* __restric
   pdl_wait();
   __shared__ double lse[G];
   __shared__ double ls_s[kFinalizeRows];   // this CTA's log-scores, for the fused block metric
-  // log-sum-exp of every head of the group from the per-chunk partials (warp g does head g)
+  // This thread's logits are requested first: they do not depend on the log-sum-exp, and the
+  // sixteen loads then overlap each other and the merge of the partials below.
+  constexpr int kPer = kFinalizeRows / kThreads;
+  const double* lu = logits + size_t(u) * G * L;
+  const int64_t j0 = int64_t(blockIdx.x) * kFinalizeRows;
+  const int64_t j1 = min(j0 + int64_t(kFinalizeRows), L);
+  double y[kPer][G];
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int64_t j = j0 + tid + i * kThreads;
+#pragma unroll
+    for (int g = 0; g < G; ++g) y[i][g] = (j < j1) ? __ldcs(lu + size_t(g) * L + j) : 0.0;
+  }
+  // log-sum-exp of every head of the group from the per-CTA partials (warp g does head g)
   {
     const int warp = tid >> 5, lane = tid & 31;
     if (warp < G) {
@@ -219,24 +235,23 @@ score_finalize_kernel(const double* __restrict__ logits, const double* __restric
   }
   __syncthreads();
   const double log_g = log(double(G));
-  const double* lu = logits + size_t(u) * G * L;
-  const int64_t j0 = int64_t(blockIdx.x) * kFinalizeRows;
-  const int64_t j1 = min(j0 + int64_t(kFinalizeRows), L);
-  for (int64_t j = j0 + tid; j < j1; j += kThreads) {
-    double y[G];
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int64_t j = j0 + tid + i * kThreads;
+    if (j >= j1) break;
     double top = -1.0e308;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      y[g] = lu[size_t(g) * L + j] - lse[g];
-      top = fmax(top, y[g]);
+      y[i][g] -= lse[g];
+      top = fmax(top, y[i][g]);
     }
     double out;
     if (G == 1) {
-      out = y[0];
+      out = y[i][0];
     } else {
       float sum = 0.f;
 #pragma unroll
-      for (int g = 0; g < G; ++g) sum += expf(float(y[g] - top));
+      for (int g = 0; g < G; ++g) sum += expf(float(y[i][g] - top));
       out = top + double(logf(sum)) - log_g;
     }
     logscore[size_t(u) * L + j] = out;
@@ -263,14 +278,20 @@ template <typename T, int D, int G>
 int launch_score(const tca_params* prm, const void* q_last, const void* K, int64_t L, double* logscore,
                  const ScoreWs& ws, const MetricOut& mo, cudaStream_t stream) {
   const int U = prm->batch * prm->n_kv_heads;
-  dim3 grid1(unsigned(ws.n_chunks), unsigned(U));
+  // One wave: as many CTAs as the GPU holds at once (four per SM at 128 registers), each with an
+  // equal share of its unit's rows, so that all of them start together and finish together; never
+  // more parts than the workspace has partials for (one per kScoreChunkRows rows).
+  const int64_t per_unit = std::max<int64_t>(1, std::min<int64_t>(ws.n_chunks, int64_t(4) * sm_count() / U));
+  const int64_t rows_per_cta = ((L + per_unit - 1) / per_unit + 31) / 32 * 32;
+  const int64_t n_parts = (L + rows_per_cta - 1) / rows_per_cta;
+  dim3 grid1(static_cast<unsigned>(n_parts), static_cast<unsigned>(U));
   int st = launch_pdl(score_logits_kernel<T, D, G>, grid1, dim3(kLogitThreads), size_t(0), stream,
                       static_cast<const T*>(q_last), static_cast<const T*>(K), L, double(prm->sm_scale), ws.logits,
-                      ws.partials, int(ws.n_chunks));
+                      ws.partials, int(n_parts), int(rows_per_cta));
   if (st != TCA_OK) return st;
   dim3 grid2(unsigned((L + kFinalizeRows - 1) / kFinalizeRows), unsigned(U));
   return launch_pdl(score_finalize_kernel<G>, grid2, dim3(kThreads), size_t(0), stream,
-                    static_cast<const double*>(ws.logits), static_cast<const double*>(ws.partials), int(ws.n_chunks), L,
+                    static_cast<const double*>(ws.logits), static_cast<const double*>(ws.partials), int(n_parts), L,
                     logscore, mo);
 }
 
