@@ -151,19 +151,6 @@ __device__ __forceinline__ unsigned long long ordered_key(double x) {
   return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// bf16 -> double by bit placement, for the two halves of a packed word.  Exact for normal
-// numbers.  Zeros and subnormals (|x| < 1.2e-38) come out as about +-5.9e-39 * (1 + m/128):
-// an absolute error below 1.2e-38 per element, invisible next to any dot product here.
-// The multiply-add form keeps half of the work off the integer ALU pipe.
-__device__ __forceinline__ double bf16_lo_to_double(uint32_t w) {
-  const uint32_t hi = (((w & 0x7FFFu) * 8192u + 0x38000000u)) | ((w << 16) & 0x80000000u);
-  return __hiloint2double(static_cast<int>(hi), 0);
-}
-__device__ __forceinline__ double bf16_hi_to_double(uint32_t w) {
-  const uint32_t hi = (((w >> 3) & 0x0FFFE000u) + 0x38000000u) | (w & 0x80000000u);
-  return __hiloint2double(static_cast<int>(hi), 0);
-}
-
 __device__ __forceinline__ float bf16_lo(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t packed) { return __uint_as_float(packed & 0xFFFF0000u); }
 
