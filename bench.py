@@ -460,8 +460,10 @@ def main():
     elt_bytes = 2 if wl.dtype == "bf16" else 4
     qo_mib = wl.batch * wl.n_q_heads * wl.L * wl.head_dim * elt_bytes / 2 ** 20
     if qo_mib > 126:
-        l2_note = (f"inputs larger than L2 (Q and O are {qo_mib:.0f} MiB each; a decode step streams the whole "
-                   "retained cache)")
+        l2_note = (f"inputs larger than L2 (Q and O are {qo_mib:.0f} MiB each; a decode step reads the whole "
+                   "retained cache, which at this size is larger than L2 too: the decode kernel asks the tiles of "
+                   "about 45 % of the L2's size to stay resident from step to step and reads those from L2, the "
+                   "rest from HBM; decode bytes in `stages` are the algorithmic ones)")
     else:
         l2_note = f"inputs smaller than L2 (Q is {qo_mib:.1f} MiB): a parity-size workload, not a bench line"
     config = {"workload": f"{wl.name}: 1 attention layer, {wl.n_q_heads}/{wl.n_kv_heads} heads, d={wl.head_dim}, "

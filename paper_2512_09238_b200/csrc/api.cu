@@ -36,6 +36,7 @@ int check_params(const tca_params* prm) {
 namespace {
 std::mutex g_device_mutex;
 int g_sm_count[kMaxDevices] = {};
+int64_t g_l2_bytes[kMaxDevices] = {};
 }  // namespace
 
 int sm_count() {
@@ -48,6 +49,17 @@ int sm_count() {
         (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
   }
   return g_sm_count[dev];
+}
+
+int64_t l2_bytes() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (g_l2_bytes[dev] == 0) {
+    int n = 0;
+    g_l2_bytes[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrL2CacheSize, dev) == cudaSuccess && n > 0) ? n : -1;
+  }
+  return g_l2_bytes[dev] > 0 ? g_l2_bytes[dev] : 0;
 }
 
 ScoreWs score_ws_layout(const tca_params* prm, int64_t L, void* ws) {

@@ -64,6 +64,7 @@ constexpr int kScoreChunkRows = 1024;  // rows of K per CTA of the logit kernel
 // Streaming multiprocessors of the current device, looked up once per device (api.cu).
 constexpr int kMaxDevices = 64;
 int sm_count();
+int64_t l2_bytes();   // L2 cache size of the current device
 
 struct ScoreWs {
   double* logits;
