@@ -183,7 +183,7 @@ class Pipeline:
             step_rows = -(-wl.L // n_ranges)
             step_rows = -(-step_rows // 128) * 128               # TCA_PREFILL_ROW_ALIGN
             cuts = list(range(0, wl.L, step_rows)) + [wl.L]
-            self.row_ranges = list(zip(cuts[:-1], cuts[1:]))[::-1]
+            self.row_ranges = list(zip(cuts[:-1], cuts[1:]))          # ascending: range i needs K, V rows below its end only
             self.ws_rows = [B.alloc_workspace(self.prm, wl.L, B.TCA_OP_PREFILL) for _ in self.row_ranges]
             self.h_Od = torch.empty_like(self.h_qd).pin_memory()
         self.launches_per_step = 4 + 1 + 1 + wl.decode_steps * 3   # score + select fused: 4, compact, prefill; append + split + combine per step
@@ -239,10 +239,11 @@ class Pipeline:
     def step_from_host(self, mark: bool = False):
         """The same step with every input in pinned host memory and every output read back.
 
-        K, V and the newest query go first (score, select and compact need nothing else); Q then
-        arrives in row ranges on a copy stream while tca_attn_prefill_rows works on the ranges
-        already there, and each finished range of O leaves on a third stream.  The last range of
-        rows (the longest) is computed first.
+        K and the newest query go first (score and select need nothing else).  V and Q then arrive
+        in row ranges, in ascending order, on a copy stream: a range of query rows attends only to
+        positions below its end, so tca_compact_kv_range gathers the retained rows of each piece of
+        V as it lands and tca_attn_prefill_rows starts on range i while the later pieces are still
+        on the bus; each finished range of O leaves on a third stream.
         """
         B, prm, L, torch = self.B, self.prm, self.L, self.torch
         cs = torch.cuda.current_stream()
@@ -252,14 +253,17 @@ class Pipeline:
         self.s_in.wait_event(start)          # the previous step has finished with these buffers
         self.s_out.wait_event(start)
         heads = [(b, h) for b in range(self.wl.batch) for h in range(self.wl.n_q_heads)]
-        ev_q = []
+        kv_heads = [(b, h) for b in range(self.wl.batch) for h in range(self.wl.n_kv_heads)]
+        ev_q, ev_v = [], []
         with torch.cuda.stream(self.s_in):
             self.Kp.copy_(self.h_Kp, non_blocking=True)
             self.q_last.copy_(self.h_q_last, non_blocking=True)
             ev_k = torch.cuda.Event(); ev_k.record(self.s_in)
-            self.Vp.copy_(self.h_Vp, non_blocking=True)
-            ev_v = torch.cuda.Event(); ev_v.record(self.s_in)
             for (r0, r1) in self.row_ranges:
+                for (b, h) in kv_heads:
+                    self.Vp[b, h, r0:r1].copy_(self.h_Vp[b, h, r0:r1], non_blocking=True)
+                e = torch.cuda.Event(); e.record(self.s_in)
+                ev_v.append(e)
                 for (b, h) in heads:
                     self.Qp[b, h, r0:r1].copy_(self.h_Qp[b, h, r0:r1], non_blocking=True)
                 e = torch.cuda.Event(); e.record(self.s_in)
@@ -273,10 +277,11 @@ class Pipeline:
         B.tca_score_select(prm, self.q_last, self.Kp, L, self.n_k, self.logscore, self.idx, self.offsets_dev, None, None,
                            self.ws_score_select)
         if mark: self._ev("t_score_select")
-        cs.wait_event(ev_v)
-        B.tca_compact_kv(prm, self.Kp, self.Vp, L, self.idx, self.offsets_dev, self.offsets, self.cache)
-        if mark: self._ev("t_compact")
+        if mark: self._ev("t_compact")          # the compaction is part of the ranges below
         for i, (r0, r1) in enumerate(self.row_ranges):
+            cs.wait_event(ev_v[i])
+            B.tca_compact_kv_range(prm, self.Kp, self.Vp, L, r0, r1, self.idx, self.offsets_dev, self.offsets,
+                                   self.cache)
             cs.wait_event(ev_q[i])
             B.tca_attn_prefill_rows(prm, self.Qp, self.Kp, self.Vp, L, r0, r1, self.cache, self.O, self.ws_rows[i])
             done = torch.cuda.Event(); done.record(cs)
@@ -655,10 +660,11 @@ def main():
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                       "prefill_ms": e2e_prefill_ms,
                       "decode_us_per_step": st_e2e["decode"] * 1e3 / wl.decode_steps if wl.decode_steps > 0 else None,
-                      "note": "pinned host buffers: K, V and the newest query copied in first; Q copied in and O copied "
-                              "back in row ranges on two copy streams while tca_attn_prefill_rows computes the "
-                              "ranges already present; decode tokens copied in, decode outputs copied back; the "
-                              "timed prefill ends when the last range of O has reached the host",
+                      "note": "pinned host buffers: K and the newest query copied in first (score + select); V and Q "
+                              "copied in, and O copied back, in ascending row ranges on two copy streams while "
+                              "tca_compact_kv_range gathers each piece of V as it lands and tca_attn_prefill_rows "
+                              "computes the ranges already present; decode tokens copied in, decode outputs copied "
+                              "back; the timed prefill ends when the last range of O has reached the host",
                       "row_ranges": len(pipe.row_ranges)}
 
     if rank == 0 and world == 1 and not args.no_calibration and wl.dtype == "bf16":

@@ -228,6 +228,20 @@ int tca_compact_kv(const tca_params* prm, const void* K, const void* V, int64_t 
                    tca_cache_desc* cache, void* stream);
 
 /*
+ * The same compaction for the retained rows whose position lies in [pos_begin, pos_end) only
+ * (0 <= pos_begin < pos_end <= L, else TCA_ERR_INVALID_ARG), for a caller whose K and V arrive
+ * in pieces: rows of K and V outside the range are not read.  Every call writes all positions
+ * and the state words (they depend on the selection alone), so after the call for positions
+ * [0, p) the cache serves tca_attn_prefill_rows for query rows below p; calls whose ranges cover
+ * [0, L), in any order, leave the cache bit-identical to one tca_compact_kv.  Other arguments
+ * and errors as tca_compact_kv.
+ */
+int tca_compact_kv_range(const tca_params* prm, const void* K, const void* V, int64_t L,
+                         int64_t pos_begin, int64_t pos_end,
+                         const int32_t* idx, const int64_t* offsets_dev, const int64_t* offsets_host,
+                         tca_cache_desc* cache, void* stream);
+
+/*
  * Sparse causal attention of the prefill, Eq. 2 / Algorithm 2 line 7.  Query i of a head
  * attends to {j <= i : j in S or j >= c_i}, c_i = min(max(0, i - w + 1), m*b): its own
  * last w keys (read from K, V) plus the selected keys before them (read from the cache's

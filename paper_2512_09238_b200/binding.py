@@ -35,7 +35,7 @@ EXPORTS = (
     "tca_cache_append", "tca_ws_status", "tca_attn_decode_static", "tca_attn_prefill_rows",
     "tca_calib_colmean", "tca_calib_score", "tca_calib_choose", "tca_calib_candidates",
     "tca_decode_static_status", "tca_selftest_wait_expiry", "tca_score_select", "tca_build_info",
-    "tca_cache_status", "tca_attn_prefill_gather",
+    "tca_cache_status", "tca_attn_prefill_gather", "tca_compact_kv_range",
 )
 
 
@@ -84,6 +84,7 @@ def load_library(path: str) -> C.CDLL:
     L.tca_score_select.argtypes = [P, vp, vp, i64, vp, C.c_int32, vp, vp, vp, vp, vp, vp, sz, vp]
     L.tca_cache_init.argtypes = [P, D, vp]
     L.tca_compact_kv.argtypes = [P, vp, vp, i64, vp, vp, vp, D, vp]
+    L.tca_compact_kv_range.argtypes = [P, vp, vp, i64, i64, i64, vp, vp, vp, D, vp]
     L.tca_attn_prefill.argtypes = [P, vp, vp, vp, i64, D, vp, vp, sz, vp]
     L.tca_attn_prefill_rows.argtypes = [P, vp, vp, vp, i64, i64, i64, D, vp, vp, sz, vp]
     L.tca_attn_prefill_gather.argtypes = [P, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]
@@ -223,6 +224,13 @@ def tca_compact_kv(prm, K, V, L, idx, offsets_dev, offsets_host, cache: "Cache",
     _check(lib().tca_compact_kv(C.byref(prm), _dev(K), _dev(V), L, _dev(idx), _dev(offsets_dev),
                                 _host(offsets_host, np.int64), C.byref(cache.desc), _stream(stream)),
            "tca_compact_kv")
+
+
+def tca_compact_kv_range(prm, K, V, L, pos_begin, pos_end, idx, offsets_dev, offsets_host, cache: "Cache",
+                         stream=None) -> None:
+    _check(lib().tca_compact_kv_range(C.byref(prm), _dev(K), _dev(V), L, pos_begin, pos_end, _dev(idx),
+                                      _dev(offsets_dev), _host(offsets_host, np.int64), C.byref(cache.desc),
+                                      _stream(stream)), "tca_compact_kv_range")
 
 
 def tca_attn_prefill(prm, Q, K, V, L, cache: "Cache", O, ws, stream=None) -> None:

@@ -83,6 +83,34 @@ def test_config3_prefill_32k_band_first():
     _check_prefill_rows(wl, data, pipe, sel, n_random=6)
 
 
+def test_the_step_from_host_buffers_equals_the_resident_step():
+    """bench.py's end-to-end step (K first, then V and Q in ascending row ranges with the compaction
+    done piece by piece as V lands, O copied back per range, decode tokens in and out) against the
+    step on resident inputs: every element of O and of the decode outputs bit for bit, starting from
+    device buffers that hold a marker instead of the inputs."""
+    wl = I.WORKLOADS["config3"].scaled(decode_steps=6)
+    data = I.generate(wl)
+    p = I.budget_table(wl)
+    ref = bench.Pipeline(wl, data, p, torch, B, host_io=False)
+    ref.step()
+    torch.cuda.synchronize()
+    pipe = bench.Pipeline(wl, data, p, torch, B, host_io=True)
+    for t in (pipe.Qp, pipe.Kp, pipe.Vp, pipe.qd, pipe.kd, pipe.vd, pipe.cache.k, pipe.cache.v, pipe.O, pipe.Od):
+        t.fill_(5.0)                                   # finite: rows past a range are masked, not skipped
+    pipe.q_last.fill_(5.0)
+    pipe.h_O.fill_(float("nan"))
+    assert len(pipe.row_ranges) > 4
+    pipe.step(host_io=True)
+    torch.cuda.synchronize()
+    for ws in pipe.ws_rows:
+        assert B.tca_ws_status(ws) == B.TCA_OK
+    assert B.tca_ws_status(pipe.ws_decode) == B.TCA_OK
+    assert torch.equal(pipe.idx, ref.idx)
+    assert torch.equal(pipe.h_O.view(torch.int16), ref.O.cpu().view(torch.int16))
+    assert torch.equal(pipe.h_Od.view(torch.int16), ref.Od.cpu().view(torch.int16))
+    assert torch.equal(pipe.cache.pos, ref.cache.pos)
+
+
 @pytest.mark.parametrize("name", ["config3", "config4"])
 def test_gather_prefill_equals_the_cache_path_at_full_size(name):
     """tca_attn_prefill_gather (selected rows fetched from K, V inside the attention kernel) over the

@@ -103,6 +103,50 @@ def test_compaction_is_bit_exact(runs, name):
             assert state[u, 2] == len(S) and state[u, 4] == wl.L - run.m * wl.block and state[u, 5] == wl.L
 
 
+@pytest.mark.parametrize("name", ["config1", "bf16_gqa4", "bf16_g7", "f32_g3_b1"])
+def test_compaction_by_position_ranges_is_bit_identical(runs, name):
+    """tca_compact_kv_range over a partition of [0, L), in a shuffled order, into a cache filled with
+    a marker: K, V, positions and state equal to one tca_compact_kv; after the call for [0, p) the
+    rows with position below p are in place and rows at or above p still hold the marker."""
+    wl, data, p, run, oracle = runs(name)
+    L = run.L
+    tk = np.tile(run.tbar, wl.batch).astype(np.int64)
+    cache = B.Cache(run.prm, np.tile(run.n_sel, wl.batch), wl.window + wl.block, tk)
+    marker = 3.0
+    cache.k.fill_(marker)
+    cache.v.fill_(marker)
+    offsets_dev = torch.from_numpy(run.offsets).cuda()
+    cuts = sorted({0, L // 5, L // 2, L - 1, L})
+    parts = [(a, b) for a, b in zip(cuts[:-1], cuts[1:]) if b > a]
+    first = parts[0]
+    B.tca_compact_kv_range(run.prm, run.dev["k"], run.dev["v"], L, first[0], first[1], run.idx, offsets_dev,
+                           run.offsets, cache)
+    torch.cuda.synchronize()
+    pos = cache.pos.cpu().numpy()
+    kc = cache.k.float().cpu().numpy()
+    ref_pos = run.cache.pos.cpu().numpy()
+    for u in range(wl.batch * wl.n_kv_heads):
+        rows = np.asarray(run.cache.unit_rows(u))
+        np.testing.assert_array_equal(pos[rows], ref_pos[rows])                 # all positions after any call
+        late = rows[ref_pos[rows] >= first[1]]
+        assert (kc[late] == marker).all()                                       # not touched yet
+    for (a, b) in parts[:0:-1]:                                                 # the rest, last range first
+        B.tca_compact_kv_range(run.prm, run.dev["k"], run.dev["v"], L, a, b, run.idx, offsets_dev, run.offsets, cache)
+    torch.cuda.synchronize()
+    raw = torch.int16 if wl.dtype == "bf16" else torch.int32
+    for u in range(wl.batch * wl.n_kv_heads):
+        rows = torch.as_tensor(np.asarray(run.cache.unit_rows(u)), device="cuda")
+        assert torch.equal(cache.k.view(raw)[rows], run.cache.k.view(raw)[rows])
+        assert torch.equal(cache.v.view(raw)[rows], run.cache.v.view(raw)[rows])
+    assert torch.equal(cache.pos, run.cache.pos)
+    assert torch.equal(cache.state, run.cache.state)
+    assert list(cache.n_global) == list(run.cache.n_global) and list(cache.n_tail) == list(run.cache.n_tail)
+    for bad in [(-1, 5), (5, 5), (0, L + 1)]:
+        with pytest.raises(B.TcaError):
+            B.tca_compact_kv_range(run.prm, run.dev["k"], run.dev["v"], L, bad[0], bad[1], run.idx, offsets_dev,
+                                   run.offsets, cache)
+
+
 def _oracle_T(run, wl, u):
     """The retained set the oracle's attention is evaluated on: the index set the GPU selected.
 
