@@ -23,6 +23,13 @@ cache_append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, co
   const int u = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, lane16 = tid & 15, grp = tid >> 4;
   int64_t* st = state + size_t(u) * TCA_STATE_WORDS;
+  // the new row is requested together with the state words (one trip to memory instead of two);
+  // head_dim <= 128 < kThreads, so a thread holds at most one element of it
+  T k_val = T(), v_val = T();
+  if (tid < D) {
+    k_val = k_new[size_t(u) * D + tid];
+    v_val = v_new[size_t(u) * D + tid];
+  }
   const int64_t seg = st[TCA_ST_SEG_START], gcap = st[TCA_ST_GLOBAL_CAP];
   const int64_t n_global = st[TCA_ST_N_GLOBAL], tail_head = st[TCA_ST_TAIL_HEAD];
   const int64_t n_tail = st[TCA_ST_N_TAIL], seq_len = st[TCA_ST_SEQ_LEN];
@@ -42,9 +49,9 @@ cache_append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, co
   // ---- append
   {
     const int64_t slot = (tail_head + n_tail) % tail_cap;
-    for (int i = tid; i < D; i += kThreads) {
-      Kc[(ring + slot) * D + i] = k_new[size_t(u) * D + i];
-      Vc[(ring + slot) * D + i] = v_new[size_t(u) * D + i];
+    if (tid < D) {
+      Kc[(ring + slot) * D + tid] = k_val;
+      Vc[(ring + slot) * D + tid] = v_val;
     }
     if (tid == 0) pos[ring + slot] = int32_t(seq_len);
   }

@@ -296,12 +296,15 @@ __global__ void __launch_bounds__(kThreads)
 decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restrict__ state, int64_t tail_cap,
                       int target, T* __restrict__ O) {
   constexpr int NW = kConsumers / 32;   // warp w merges partials w, w + NW, ...; a lane owns 4 outputs
-  pdl_wait();                 // the partials come from the split kernel
-  pdl_launch_dependents();
+  // The state words were written before the split kernel started (it triggered this launch only
+  // after its own dependency wait had returned), so where this CTA's partials lie is worked out
+  // while the split kernel is still streaming; only the partials themselves need the wait.
   const int g = blockIdx.x, u = blockIdx.y;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int n_chunks = n_parts(uv.len(), target);
   const int base_slot = partial_base(state, u, target);
+  pdl_wait();                 // the partials come from the split kernel
+  pdl_launch_dependents();
   const int tid = threadIdx.x;
   if (tid >= kConsumers) return;
   const float* base = partial + size_t(base_slot) * G * (D + 2) + size_t(g) * (D + 2);
