@@ -100,6 +100,26 @@ def test_prefill_refuses_a_zero_window_before_touching_anything():
     assert L.tca_attn_prefill(ctypes.byref(w1), None, None, None, 2048, None, None, None, 0, None) == B.TCA_ERR_INVALID_ARG
 
 
+def test_gather_prefill_and_ranged_compaction_validate_their_arguments_on_the_host():
+    """The two entry points added beside tca_attn_prefill_rows and tca_compact_kv refuse what they
+    do not support, and bad ranges, before anything touches the device."""
+    L = B.lib()
+    f32 = B.make_params(1, 8, 8, 64, 32, 128, dtype=B.TCA_F32)
+    assert L.tca_attn_prefill_gather(ctypes.byref(f32), None, None, None, 2048, 0, 2048, None, None, None, None, 0,
+                                     None) == B.TCA_ERR_UNSUPPORTED          # tensor-core kernel only: bf16
+    bf = B.make_params(1, 8, 8, 64, 32, 128, dtype=B.TCA_BF16)
+    simt = B.make_params(1, 8, 8, 64, 32, 128, dtype=B.TCA_BF16, flags=B.TCA_FLAG_PREFILL_SIMT)
+    assert L.tca_attn_prefill_gather(ctypes.byref(simt), None, None, None, 2048, 0, 2048, None, None, None, None, 0,
+                                     None) == B.TCA_ERR_UNSUPPORTED
+    assert L.tca_attn_prefill_gather(ctypes.byref(bf), None, None, None, 2048, 0, 2048, None, None, None, None, 0,
+                                     None) == B.TCA_ERR_INVALID_ARG          # NULL buffers
+    w0 = B.make_params(1, 8, 8, 64, 32, 0, dtype=B.TCA_BF16)
+    assert L.tca_attn_prefill_gather(ctypes.byref(w0), None, None, None, 2048, 0, 2048, None, None, None, None, 0,
+                                     None) == B.TCA_ERR_UNSUPPORTED          # window >= 1, as for the other prefills
+    assert L.tca_compact_kv_range(ctypes.byref(bf), None, None, 2048, 0, 2048, None, None, None, None,
+                                  None) == B.TCA_ERR_INVALID_ARG
+
+
 def test_static_decode_limit_formula_is_the_workspace_size():
     """The limit documented for tca_attn_decode_static is tca_workspace_bytes for TCA_OP_DECODE."""
     def up(x):
