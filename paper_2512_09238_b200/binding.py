@@ -110,7 +110,8 @@ def lib() -> C.CDLL:
     """The loaded library; raises if it has not been built (no fallback exists)."""
     global _lib
     if _lib is None:
-        _lib = load_library(LIB_PATH)
+        # TCA_LIBRARY names another build of the same library, e.g. the range-checked libtca_dbg.so
+        _lib = load_library(os.environ.get("TCA_LIBRARY") or LIB_PATH)
     return _lib
 
 
