@@ -8,7 +8,9 @@
  *     cache, workspace) are allocated and freed by the caller; the library calls no
  *     allocator.  What it keeps between calls is limited to: the built-in scratch array of
  *     tca_attn_decode_static (and its per-device address), a small cache of encoded TMA
- *     tensor maps keyed by buffer address and shape, and per-device constants (SM count).
+ *     tensor maps keyed by buffer address and shape, and per-device constants (SM count,
+ *     L2 cache size).  The bf16 decode kernel asks the L2 to keep part of the cache it reads
+ *     (eviction-priority hints on its loads; nothing is set on the device or the context).
  *   - Tensors are row-major with the head dimension contiguous:
  *       Q [batch, n_q_heads, L, head_dim]      K, V [batch, n_kv_heads, L, head_dim]
  *     A "unit" is one (sequence, KV head) pair, u = seq * n_kv_heads + kv_head; the G =
