@@ -111,7 +111,9 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       // The cache is read again by the next step, and its rows stay where they are: l2_keep of every
       // 64 tiles (by address, hence the same ones every step) ask to stay in L2, the others to be
       // evicted first, so that the part of the cache that fits keeps being served from L2 instead of
-      // the whole of it sweeping through.
+      // the whole of it sweeping through.  The choice goes by the bit-reversed tile index, which
+      // spreads the resident tiles evenly (every fourth tile for a quarter), so that every CTA's
+      // slice holds the same share of them and the CTAs keep finishing together.
       const uint64_t pol_keep = ptx::l2_policy_evict_last(), pol_stream = ptx::l2_policy_evict_first();
       while (done < n_rows) {
         const int64_t r = row0 + done;
@@ -130,7 +132,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           uint8_t* dst = ring_buf + (n % kStages) * Ring::kTileBytes;
           for (int box = 0; box < D / 64; ++box)
             ptx::tma_load_2d_hint(dst + box * kBoxBytes, kv ? &map_v : &map_k, box * 64, y, &ring.full[n % kStages],
-                                  (((y >> 7) & 63) < l2_keep) ? pol_keep : pol_stream);
+                                  (int(__brev(unsigned(y >> 7)) >> 26) < l2_keep) ? pol_keep : pol_stream);
         }
         done += cnt;
       }
