@@ -53,7 +53,7 @@ template <typename T, int D, int G>
 __global__ void __maxnreg__(112)
 decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* __restrict__ Vc,
                     const int64_t* __restrict__ state, int64_t tail_cap, float scale_log2e, int target,
-                    float* __restrict__ partial, int* __restrict__ status) {
+                    float* __restrict__ partial, int* __restrict__ status, int n_units) {
   using Cfg = DecCfg<G>;
   using Ring = DecRing<T, D>;
   constexpr int EPL = D / 16;
@@ -61,17 +61,17 @@ decode_split_kernel(const T* __restrict__ q, const T* __restrict__ Kc, const T* 
   constexpr int kStages = Ring::kStages;
   pdl_wait();
   pdl_launch_dependents();
-  const int u = blockIdx.y;
-  const int part_idx = blockIdx.x;
+  __shared__ SliceId slice_slot;
+  const SliceId slice = find_slice(state, n_units, target, &slice_slot);
+  if (slice.u < 0) return;
+  const int u = slice.u, part_idx = slice.part, np = slice.np;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int64_t len = uv.len();
-  const int np = n_parts(len, target);
-  if (part_idx >= np) return;
   const int64_t row0 = slice_begin(len, np, part_idx);
   const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
   const int n_super = (n_rows + kSuperRows - 1) / kSuperRows;
   const int tid = threadIdx.x, lane16 = tid & 15, grp = tid >> 4, warp = tid >> 5;
-  const int base_slot = partial_base(state, u, target);
+  const int base_slot = slice.base_slot;
 
   extern __shared__ uint8_t dec_smem_raw[];
   uint8_t* ring_buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dec_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -360,14 +360,13 @@ decode_combine_kernel(const float* __restrict__ partial, const int64_t* __restri
 }
 
 // Rows per CTA: enough CTAs for two per SM, at least one softmax round each.
-inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_sm, int64_t* max_len_out) {
+inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_sm, int64_t* n_slices_out) {
   int64_t total = 0, max_len = 0;
   for (int64_t u = 0; u < U; ++u) {
     const int64_t len = c->n_global[u] + c->n_tail[u];
     total += len;
     max_len = len > max_len ? len : max_len;
   }
-  *max_len_out = max_len;
   const int sms = sm_count();
   // Smallest slice length for which the slices of all units fit the resident CTAs in one
   // wave: with one slice more than that, the extra CTA starts only after another one ends.
@@ -386,12 +385,13 @@ inline int decode_target_rows(const tca_cache_desc* c, int64_t U, int ctas_per_s
       if (count(mid) <= slots) hi = mid; else lo = mid + 1;
     }
   }
+  *n_slices_out = count(lo);   // CTAs of the attention kernel: one per slice
   return int(lo);
 }
 
 template <typename T, int D, int G>
 int launch_decode(const tca_params* prm, const void* q, const tca_cache_desc* c, void* O, const DecodeWs& ws,
-                  int64_t max_len, int target, cudaStream_t stream) {
+                  int64_t n_slices, int target, cudaStream_t stream) {
   using Ring = DecRing<T, D>;
   const int U = prm->batch * prm->n_kv_heads;
   const float scale_log2e = prm->sm_scale * 1.4426950408889634f;
@@ -399,12 +399,12 @@ int launch_decode(const tca_params* prm, const void* q, const tca_cache_desc* c,
   TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Ring::kSmemBytes));
   int st;
   if constexpr (sizeof(T) == 2) {
-    st = launch_decode_mma<D>(prm, q, c, ws, max_len, target, stream);   // tensor-pipe kernel for bf16
+    st = launch_decode_mma<D>(prm, q, c, ws, n_slices, target, stream);   // tensor-pipe kernel for bf16
   } else {
-    dim3 grid(unsigned((max_len + target - 1) / target), unsigned(U));
+    dim3 grid(static_cast<unsigned>(n_slices));   // one CTA per slice, none idle (see find_slice)
     kern<<<grid, kThreads, Ring::kSmemBytes, stream>>>(
         static_cast<const T*>(q), static_cast<const T*>(c->k), static_cast<const T*>(c->v), c->state,
-        c->tail_cap, scale_log2e, target, ws.partial, ws.status);
+        c->tail_cap, scale_log2e, target, ws.partial, ws.status, int(U));
     st = check_launch();
   }
   if (st != TCA_OK) return st;
@@ -415,16 +415,16 @@ int launch_decode(const tca_params* prm, const void* q, const tca_cache_desc* c,
 
 template <typename T, int D>
 int dispatch_group(int G, const tca_params* prm, const void* q, const tca_cache_desc* c, void* O,
-                   const DecodeWs& ws, int64_t max_len, int target, cudaStream_t s) {
+                   const DecodeWs& ws, int64_t n_slices, int target, cudaStream_t s) {
   switch (G) {
-    case 1: return launch_decode<T, D, 1>(prm, q, c, O, ws, max_len, target, s);
-    case 2: return launch_decode<T, D, 2>(prm, q, c, O, ws, max_len, target, s);
-    case 3: return launch_decode<T, D, 3>(prm, q, c, O, ws, max_len, target, s);
-    case 4: return launch_decode<T, D, 4>(prm, q, c, O, ws, max_len, target, s);
-    case 5: return launch_decode<T, D, 5>(prm, q, c, O, ws, max_len, target, s);
-    case 6: return launch_decode<T, D, 6>(prm, q, c, O, ws, max_len, target, s);
-    case 7: return launch_decode<T, D, 7>(prm, q, c, O, ws, max_len, target, s);
-    case 8: return launch_decode<T, D, 8>(prm, q, c, O, ws, max_len, target, s);
+    case 1: return launch_decode<T, D, 1>(prm, q, c, O, ws, n_slices, target, s);
+    case 2: return launch_decode<T, D, 2>(prm, q, c, O, ws, n_slices, target, s);
+    case 3: return launch_decode<T, D, 3>(prm, q, c, O, ws, n_slices, target, s);
+    case 4: return launch_decode<T, D, 4>(prm, q, c, O, ws, n_slices, target, s);
+    case 5: return launch_decode<T, D, 5>(prm, q, c, O, ws, n_slices, target, s);
+    case 6: return launch_decode<T, D, 6>(prm, q, c, O, ws, n_slices, target, s);
+    case 7: return launch_decode<T, D, 7>(prm, q, c, O, ws, n_slices, target, s);
+    case 8: return launch_decode<T, D, 8>(prm, q, c, O, ws, n_slices, target, s);
     default: return TCA_ERR_UNSUPPORTED;
   }
 }
@@ -445,17 +445,17 @@ extern "C" int tca_attn_decode(const tca_params* prm, const void* q, const tca_c
   TCA_CHECK_ARG(c->n_units == U && U <= 65535);
   DecodeWs lay = decode_ws_layout(prm, c->rows_total, U, ws);
   if (ws_bytes < lay.bytes) return TCA_ERR_WORKSPACE;
-  int64_t max_len = 0;
-  const int target = decode_target_rows(c, U, prm->dtype == TCA_BF16 ? 1 : 2, &max_len);
-  TCA_CHECK_ARG(max_len >= 1);
+  int64_t n_slices = 0;
+  const int target = decode_target_rows(c, U, prm->dtype == TCA_BF16 ? 1 : 2, &n_slices);
+  TCA_CHECK_ARG(n_slices >= 1);
   const int G = prm->n_q_heads / prm->n_kv_heads;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (prm->dtype == TCA_BF16) {
-    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, target, s);
-    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, target, s);
+    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, n_slices, target, s);
+    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, n_slices, target, s);
   }
-  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, target, s);
-  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, target, s);
+  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, n_slices, target, s);
+  return dispatch_group<float, 64>(G, prm, q, c, O, lay, n_slices, target, s);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -507,17 +507,17 @@ extern "C" int tca_attn_decode_static(const tca_params* prm, const void* q, cons
   st = static_scratch(&scratch);
   if (st != TCA_OK) return st;
   lay = decode_ws_layout(prm, c->rows_total, U, scratch);
-  int64_t max_len = 0;
-  const int target = decode_target_rows(c, U, prm->dtype == TCA_BF16 ? 1 : 2, &max_len);
-  TCA_CHECK_ARG(max_len >= 1);
+  int64_t n_slices = 0;
+  const int target = decode_target_rows(c, U, prm->dtype == TCA_BF16 ? 1 : 2, &n_slices);
+  TCA_CHECK_ARG(n_slices >= 1);
   const int G = prm->n_q_heads / prm->n_kv_heads;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (prm->dtype == TCA_BF16) {
-    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, max_len, target, s);
-    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, max_len, target, s);
+    if (prm->head_dim == 128) return dispatch_group<__nv_bfloat16, 128>(G, prm, q, c, O, lay, n_slices, target, s);
+    return dispatch_group<__nv_bfloat16, 64>(G, prm, q, c, O, lay, n_slices, target, s);
   }
-  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, max_len, target, s);
-  return dispatch_group<float, 64>(G, prm, q, c, O, lay, max_len, target, s);
+  if (prm->head_dim == 128) return dispatch_group<float, 128>(G, prm, q, c, O, lay, n_slices, target, s);
+  return dispatch_group<float, 64>(G, prm, q, c, O, lay, n_slices, target, s);
 }
 
 extern "C" int tca_decode_static_status(void* stream) {

@@ -55,4 +55,50 @@ __device__ __forceinline__ int partial_base(const int64_t* state, int u, int tar
   return part;
 }
 
+// Which slice a CTA of the attention kernels works on.  blockIdx.x counts the slices of all units,
+// unit after unit, and exactly as many CTAs are launched as there are slices: a CTA without work
+// would still hold its SM until its dependency wait returns, and the slices behind it in launch
+// order would start that much later (with a grid of units x longest-unit-slices, 124 of 272 CTAs
+// were idle at the benchmark's mix of budgets and the last slices started 4-5 us late).
+struct SliceId {
+  int u;           // unit, -1 if blockIdx.x lies beyond the last slice
+  int part;        // slice within the unit
+  int np;          // slices of the unit
+  int base_slot;   // slices of all earlier units = first partial slot of this unit
+};
+// Called by every thread of the CTA (it contains a CTA-wide barrier); warp 0 does the search, 32
+// units per round with a warp scan.
+__device__ __forceinline__ SliceId find_slice(const int64_t* state, int n_units, int target, SliceId* shared_slot) {
+  if (threadIdx.x < 32) {
+    const int lane = int(threadIdx.x), lin = int(blockIdx.x);
+    int offset = 0;
+    bool found = false;
+    for (int v0 = 0; v0 < n_units && !found; v0 += 32) {
+      const int v = v0 + lane;
+      int npv = 0;
+      if (v < n_units) {
+        const int64_t* st = state + size_t(v) * TCA_STATE_WORDS;
+        npv = n_parts(st[TCA_ST_N_GLOBAL] + st[TCA_ST_N_TAIL], target);
+      }
+      int incl = npv;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+      }
+      const unsigned hit = __ballot_sync(0xffffffffu, lin < offset + incl);
+      if (hit) {
+        const int l = __ffs(hit) - 1;
+        const int excl = __shfl_sync(0xffffffffu, incl - npv, l), npl = __shfl_sync(0xffffffffu, npv, l);
+        if (lane == 0) *shared_slot = SliceId{v0 + l, lin - offset - excl, npl, offset + excl};
+        found = true;
+      }
+      offset += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (!found && lane == 0) *shared_slot = SliceId{-1, 0, 0, 0};
+  }
+  __syncthreads();
+  return *shared_slot;
+}
+
 }  // namespace tca

@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1)
 decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                   const __nv_bfloat16* __restrict__ q, const int64_t* __restrict__ state, int64_t tail_cap,
                   int G, float scale_log2e, int target, float* __restrict__ partial, int* __restrict__ status,
-                  int l2_keep) {
+                  int l2_keep, int n_units) {
   using Ring = MmaRing<D>;
   constexpr int kStages = Ring::kStages;
   constexpr int ND = D / 8;     // n8 tiles across the head dimension
@@ -83,6 +83,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   uint8_t* ring_buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dmma_smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ BulkRing<kStages> ring;
   __shared__ int abort_word;
+  __shared__ SliceId slice_slot;
   __shared__ float s_m[kMmaConsumers / 32][kMaxGroup], s_l[kMmaConsumers / 32][kMaxGroup];
   volatile int* abort_flag = &abort_word;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -96,11 +97,11 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   __syncthreads();
   pdl_wait();                 // the cache state and rows come from the kernels before this one
   pdl_launch_dependents();
-  const int u = blockIdx.y, part_idx = blockIdx.x;
+  const SliceId slice = find_slice(state, n_units, target, &slice_slot);
+  if (slice.u < 0) return;
+  const int u = slice.u, part_idx = slice.part, np = slice.np;
   const UnitView uv = load_unit(state, u, tail_cap);
   const int64_t len = uv.len();
-  const int np = n_parts(len, target);
-  if (part_idx >= np) return;
   const int64_t row0 = slice_begin(len, np, part_idx);
   const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
 
@@ -141,7 +142,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   }
 
   // --------------------------------------------------------------- consumers
-  const int base_slot = partial_base(state, u, target);
+  const int base_slot = slice.base_slot;
   const int gq = lane >> 2, kq = (lane & 3) * 2;   // accumulator row (query head) and column pair
   // Q as the A operand, one k16 chunk of the head dimension per entry (rows >= G are zero)
   uint32_t qa[KC][2];
@@ -328,7 +329,7 @@ bool cache_map(const void* base, int64_t rows, int D, CUtensorMap* out) {
 
 template <int D>
 int launch_decode_mma(const tca_params* prm, const void* q, const tca_cache_desc* c, const DecodeWs& ws,
-                      int64_t max_len, int target, cudaStream_t stream) {
+                      int64_t n_slices, int target, cudaStream_t stream) {
   using Ring = MmaRing<D>;
   CUtensorMap mk, mv;
   if (!cache_map(c->k, c->rows_total, D, &mk) || !cache_map(c->v, c->rows_total, D, &mv)) return TCA_ERR_CUDA;
@@ -342,10 +343,10 @@ int launch_decode_mma(const tca_params* prm, const void* q, const tca_cache_desc
   const int l2_keep = keep >= 1.0 ? 64 : int(keep * 64.0 + 0.5);
   auto kern = decode_mma_kernel<D>;
   TCA_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Ring::kSmemBytes));
-  dim3 grid(unsigned((max_len + target - 1) / target), unsigned(U));
+  dim3 grid(static_cast<unsigned>(n_slices));   // one CTA per slice, none idle (see find_slice)
   return launch_pdl(kern, grid, dim3(kMmaThreads), size_t(Ring::kSmemBytes), stream, mk, mv,
                     static_cast<const __nv_bfloat16*>(q), static_cast<const int64_t*>(c->state), c->tail_cap, G,
-                    prm->sm_scale * 1.4426950408889634f, target, ws.partial, ws.status, l2_keep);
+                    prm->sm_scale * 1.4426950408889634f, target, ws.partial, ws.status, l2_keep, U);
 }
 
 template int launch_decode_mma<64>(const tca_params*, const void*, const tca_cache_desc*, const DecodeWs&, int64_t,
