@@ -65,10 +65,12 @@ struct SliceId {
   int part;        // slice within the unit
   int np;          // slices of the unit
   int base_slot;   // slices of all earlier units = first partial slot of this unit
+  UnitView uv;     // the unit's state words, fetched in the same trip to memory as the search
 };
 // Called by every thread of the CTA (it contains a CTA-wide barrier); warp 0 does the search, 32
 // units per round with a warp scan.
-__device__ __forceinline__ SliceId find_slice(const int64_t* state, int n_units, int target, SliceId* shared_slot) {
+__device__ __forceinline__ SliceId find_slice(const int64_t* state, int n_units, int target, int64_t tail_cap,
+                                              SliceId* shared_slot) {
   if (threadIdx.x < 32) {
     const int lane = int(threadIdx.x), lin = int(blockIdx.x);
     int offset = 0;
@@ -76,9 +78,10 @@ __device__ __forceinline__ SliceId find_slice(const int64_t* state, int n_units,
     for (int v0 = 0; v0 < n_units && !found; v0 += 32) {
       const int v = v0 + lane;
       int npv = 0;
+      UnitView mine{};
       if (v < n_units) {
-        const int64_t* st = state + size_t(v) * TCA_STATE_WORDS;
-        npv = n_parts(st[TCA_ST_N_GLOBAL] + st[TCA_ST_N_TAIL], target);
+        mine = load_unit(state, v, tail_cap);
+        npv = n_parts(mine.len(), target);
       }
       int incl = npv;
 #pragma unroll
@@ -90,12 +93,12 @@ __device__ __forceinline__ SliceId find_slice(const int64_t* state, int n_units,
       if (hit) {
         const int l = __ffs(hit) - 1;
         const int excl = __shfl_sync(0xffffffffu, incl - npv, l), npl = __shfl_sync(0xffffffffu, npv, l);
-        if (lane == 0) *shared_slot = SliceId{v0 + l, lin - offset - excl, npl, offset + excl};
+        if (lane == l) *shared_slot = SliceId{v, lin - offset - excl, npl, offset + excl, mine};
         found = true;
       }
       offset += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (!found && lane == 0) *shared_slot = SliceId{-1, 0, 0, 0};
+    if (!found && lane == 0) shared_slot->u = -1;
   }
   __syncthreads();
   return *shared_slot;

@@ -97,10 +97,10 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   __syncthreads();
   pdl_wait();                 // the cache state and rows come from the kernels before this one
   pdl_launch_dependents();
-  const SliceId slice = find_slice(state, n_units, target, &slice_slot);
+  const SliceId slice = find_slice(state, n_units, target, tail_cap, &slice_slot);
   if (slice.u < 0) return;
   const int u = slice.u, part_idx = slice.part, np = slice.np;
-  const UnitView uv = load_unit(state, u, tail_cap);
+  const UnitView uv = slice.uv;
   const int64_t len = uv.len();
   const int64_t row0 = slice_begin(len, np, part_idx);
   const int n_rows = int(slice_begin(len, np, part_idx + 1) - row0);
