@@ -32,7 +32,8 @@
 // maximum; then the exponentials in eight groups of 16, each group's packed bf16 results stored to
 // TMEM only after the next group's arithmetic has been issued, so the MUFU, which limits this
 // phase (one ex2 per score is as many MUFU clocks as the two products of the tile are tensor
-// clocks), is never left to drain.  P reaches the PV product in two halves of 64 keys, each
+// clocks), is never left to drain.  P reaches the PV product in two parts (96 keys, then 32: the
+// less is left to issue after the last announcement, the sooner the next S can follow), each
 // announced by one arrival per warp.  O stays in TMEM and is rescaled lazily: only when a row
 // maximum grew by more than 2^8 since the last rescale.
 // CTAs are ordered unit-major so that the CTAs resident at one time read the same one or two
@@ -58,7 +59,8 @@ constexpr int kRing = 5;                // K/V tiles in shared memory
 constexpr int kPairs = 3;               // (V_t, K_t+1) barrier pairs that can be in flight
 constexpr int kHalfBytes = 128 * 128;   // 128 rows x 128 bytes (64 bf16): one swizzled box
 constexpr float kRescaleThreshold = 8.f;
-constexpr int kPHalves = 2;             // P reaches the PV product in two halves of 64 keys
+constexpr int kPHalves = 2;             // P reaches the PV product in two parts
+constexpr int kPSplit = 6;              // k-steps (16 keys each) in the first part: 96 keys, then 32
 
 template <int D>
 struct TcCfg {
@@ -340,20 +342,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
       };
       // O += P V with P read from TMEM (packed bf16 over the first 64 columns of S): the A operand
-      // costs no shared-memory bandwidth.  The first four k-steps (64 keys) go as soon as the first
-      // half of P is announced, while the softmax warps still work on the second half.
+      // costs no shared-memory bandwidth.  The first kPSplit k-steps go as soon as the first
+      // part of P is announced, while the softmax warps still work on the rest.
       auto issue_PV = [&](int h, int slot, bool acc, uint32_t parity) -> bool {
         const uint64_t b0 = dv + uint64_t(uint32_t(slot * Cfg::kKV) >> 4);
         const uint32_t d = tmem_base + Cfg::colO(h);
         const uint32_t a = tmem_base + Cfg::colP(h);
-        constexpr int kPer = BN / 16 / kPHalves;
 #pragma unroll
         for (int c = 0; c < kPHalves; ++c) {
           if (!wait(&bars[BAR_P + h * kPHalves + c], parity)) return false;
           ptx::tc_fence_after();
 #pragma unroll
-          for (int k2 = 0; k2 < kPer; ++k2) {
-            const int kk = c * kPer + k2;
+          for (int kk = (c == 0 ? 0 : kPSplit); kk < (c == 0 ? kPSplit : BN / 16); ++kk) {
             ptx::umma_ts_elect(d, a + uint32_t(kk * 8), b0 + uint32_t((kk * 2048) >> 4), idescPV,
                                (acc || kk > 0) ? 1u : 0u);
           }
@@ -485,7 +485,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               sum2[j & 1] = ptx::add2(sum2[j & 1], ptx::pack2(el, eh));
               v[j] = ptx::pack_bf16x2(el, eh);   // entry j is never read again (j <= 2j)
             }
-            if (g == 5) {   // groups 0-3 (the first 64 keys) were stored at least one group ago
+            if (g == kPSplit + 1) {   // groups 0 .. kPSplit-1 (the first 96 keys) were stored at least one group ago
               ptx::tc_wait_st();
               ptx::tc_fence_before();
               __syncwarp();
