@@ -446,7 +446,7 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the 100 %-budget comparison run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="config5: skip the five-budget sweep")
-    ap.add_argument("--prefill-order", default="global", choices=["global", "band"],
+    ap.add_argument("--prefill-order", default="band", choices=["global", "band"],
                     help="key-tile order of the prefill in the timed run: selected keys first, or the window band first "
                          "(the band needs no selection, so the prefill then starts under score/select/compact)")
     ap.add_argument("--no-order-compare", action="store_true", help="skip timing the other prefill order")
