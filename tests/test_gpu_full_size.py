@@ -83,7 +83,8 @@ def test_config3_prefill_32k_band_first():
     _check_prefill_rows(wl, data, pipe, sel, n_random=6)
 
 
-def test_the_step_from_host_buffers_equals_the_resident_step():
+@pytest.mark.parametrize("flags", [0, B.TCA_FLAG_PREFILL_BAND_FIRST])
+def test_the_step_from_host_buffers_equals_the_resident_step(flags):
     """bench.py's end-to-end step (K first, then V and Q in ascending row ranges with the compaction
     done piece by piece as V lands, O copied back per range, decode tokens in and out) against the
     step on resident inputs: every element of O and of the decode outputs bit for bit, starting from
@@ -91,10 +92,10 @@ def test_the_step_from_host_buffers_equals_the_resident_step():
     wl = I.WORKLOADS["config3"].scaled(decode_steps=6)
     data = I.generate(wl)
     p = I.budget_table(wl)
-    ref = bench.Pipeline(wl, data, p, torch, B, host_io=False)
+    ref = bench.Pipeline(wl, data, p, torch, B, host_io=False, flags=flags)
     ref.step()
     torch.cuda.synchronize()
-    pipe = bench.Pipeline(wl, data, p, torch, B, host_io=True)
+    pipe = bench.Pipeline(wl, data, p, torch, B, host_io=True, flags=flags)
     for t in (pipe.Qp, pipe.Kp, pipe.Vp, pipe.qd, pipe.kd, pipe.vd, pipe.cache.k, pipe.cache.v, pipe.O, pipe.Od):
         t.fill_(5.0)                                   # finite: rows past a range are masked, not skipped
     pipe.q_last.fill_(5.0)
