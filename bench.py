@@ -235,7 +235,7 @@ class Pipeline:
         assert B.tca_ws_status(self.ws_prefill) == B.TCA_OK
         sel, pf = float(np.median(ms_sel)), float(np.median(ms_pf))
         return {"score_select_ms": sel, "prefill_ms": pf, "total_ms": sel + pf, "reps": reps,
-                "note": "tca_attn_prefill_gather: selected rows fetched from K, V by TMA row gathers in the producer"}
+                "note": "tca_attn_prefill_gather: selected rows fetched from K, V by the kernel's two producer warps (16-byte asynchronous copies)"}
 
     def step_from_host(self, mark: bool = False):
         """The same step with every input in pinned host memory and every output read back.

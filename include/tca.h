@@ -278,7 +278,9 @@ int tca_attn_prefill_rows(const tca_params* prm, const void* Q, const void* K, c
  * themselves, by index, inside the attention kernel (Appendix C, "Memory Access Optimization":
  * gathering fused into the consumer instead of a separate compaction pass).  For a caller that
  * only prefills, or that builds the decode cache later: no tca_compact_kv, no cache memory.
- * O is bit-identical to tca_compact_kv + tca_attn_prefill_rows over the same selection.
+ * O is bit-identical to tca_compact_kv + tca_attn_prefill_rows over the same selection; the
+ * call takes about 1.5 times as long as the prefill over a compacted cache (every block of the
+ * grid gathers its rows again), so it pays only where the cache memory cannot be afforded.
  *   idx, offsets_dev  DEVICE, as written by / given to tca_select: unit u's selected positions
  *                     are idx[offsets_dev[u] .. offsets_dev[u+1]), ascending; not modified
  *   row_begin, row_end  as in tca_attn_prefill_rows ([0, L) for the whole prefill)

@@ -18,7 +18,8 @@
 // and waits for them (griddepcontrol.wait) only where it first touches the cache.
 //
 // Warp roles (384 threads = 3 warpgroups): warp 0 = TMA producer (one lane), warp 1 = MMA issuer,
-// warp 2 = geometry of the global range (a warp-wide search at the start), warp 3 idle;
+// warp 2 = geometry of the global range (a warp-wide search at the start), warp 3 idle (when the
+// selected rows are gathered from K and V instead of read from the cache: second producer);
 // warps 4-7 / 8-11 = softmax of head 0 / head 1 (one thread per
 // query row = one TMEM lane).  The first warpgroup hands most of its registers to the other two
 // (setmaxnreg), so that a softmax thread can hold its row of 128 scores without spilling.
@@ -120,9 +121,9 @@ __device__ __forceinline__ int lower_bound_pos_warp(const int32_t* pos, int lo, 
 }
 
 // kGather: the selected keys are not read from a compacted cache but fetched from K and V
-// themselves, row by row, by the producer (tile::gather4); `pos` is then the index set that the
-// selection wrote, `state` its per-unit offsets, and map_ck / map_cv are row-gather maps over the
-// flattened K and V.
+// themselves (Kraw, Vraw), row by row, by two producer warps with 16-byte asynchronous copies that
+// they place into the swizzled tile themselves; `pos` is then the index set that the selection wrote,
+// `state` its per-unit offsets, and map_ck / map_cv are not used.
 template <int D, bool kGather>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -130,7 +131,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                   const __grid_constant__ CUtensorMap map_cv, const int32_t* __restrict__ pos,
                   const int64_t* __restrict__ state, int64_t L, int n_q_heads, int n_kv_heads, int window,
                   int64_t mb, float scale_log2e, __nv_bfloat16* __restrict__ O, int* __restrict__ status,
-                  int n_qtiles, int pairs_per_unit, int tile0, int band_first) {
+                  int n_qtiles, int pairs_per_unit, int tile0, int band_first,
+                  const __nv_bfloat16* __restrict__ Kraw, const __nv_bfloat16* __restrict__ Vraw) {
   using Cfg = TcCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -162,10 +164,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
   if (tid == 0) {
     ptx::mbar_init(&bars[BAR_Q], 1);
-    ptx::mbar_init(&bars[BAR_K0_FULL], 1);
+    ptx::mbar_init(&bars[BAR_K0_FULL], kGather ? 32 : 1);   // gathering: every producer lane arrives
     ptx::mbar_init(&bars[BAR_K0_EMPTY], 1);
     ptx::mbar_init(&bars[BAR_GEO], 1);
-    for (int i = 0; i < kPairs; ++i) { ptx::mbar_init(&bars[BAR_FULL + i], 2); ptx::mbar_init(&bars[BAR_EMPTY + i], 1); }
+    for (int i = 0; i < kPairs; ++i) {
+      ptx::mbar_init(&bars[BAR_FULL + i], kGather ? 64 : 2);
+      ptx::mbar_init(&bars[BAR_EMPTY + i], 1);
+    }
     for (int h = 0; h < 2; ++h) {
       ptx::mbar_init(&bars[BAR_S + h], 1);
       for (int c = 0; c < kPHalves; ++c) ptx::mbar_init(&bars[BAR_P + h * kPHalves + c], 4);   // one arrival per warp
@@ -237,10 +242,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         __threadfence_block();
         ptx::mbar_arrive(&bars[BAR_GEO]);
       }
-    } else if (warp == 0) {
-      // ------------------------------------------------------------- TMA producer
-      // One lane issues the box loads.  Row gathers are issued by the whole warp, a lane for every
-      // four rows of the tile, so there all lanes walk the loop and every wait is made warp-uniform.
+    } else if (warp == 0 || (kGather && warp == 3)) {
+      // ------------------------------------------------------------- producer
+      // One lane of warp 0 issues the box loads.  Row gathers take a whole warp per tile (and one
+      // warp cannot keep up with the tensor pipe), so when gathering warp 0 brings the K tiles and
+      // warp 3 the V tiles; all their lanes walk the loop and every wait is made warp-uniform.
+      const bool do_k = !kGather || warp == 0, do_v = !kGather || warp == 3;
       if (kGather || lane == 0) {
         auto pwait = [&](uint64_t* bar, uint32_t parity) -> bool {
           const bool r = ptx::mbar_wait(bar, parity, abort_flag);
@@ -249,7 +256,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         auto plearn = [&]() -> bool {
           if constexpr (kGather) return learn_geometry_warp(); else return learn_geometry();
         };
-        if (lane == 0) {
+        if (lane == 0 && do_k) {
           ptx::mbar_arrive_expect_tx(&bars[BAR_Q], uint32_t(nh * Cfg::kQ));
           for (int h = 0; h < nh; ++h)
             for (int half = 0; half < Cfg::NH; ++half)
@@ -265,8 +272,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           if (t >= geo.n_a && !geo_known) { ok = plearn(); if (!ok) break; }
           if (t >= geo.n_a + geo.n_b) {
             // past the last tile: the last pair holds V only, its barrier still expects two arrivals
-            if (!is_v && t > 0 && lane == 0) ptx::mbar_arrive(&bars[BAR_FULL + (t - 1) % kPairs]);
+            if (!is_v && t > 0 && do_k && (kGather || lane == 0)) ptx::mbar_arrive(&bars[BAR_FULL + (t - 1) % kPairs]);
             break;
+          }
+          if (is_v ? !do_v : !do_k) continue;                  // the other producer warp's tile
+          // The row numbers of a gathered tile are requested before the wait for the ring slot, which
+          // hides their latency.  Row r of the tile is the unit's selected key number index(t)*128 + r;
+          // a tile that reaches past the keys visible to this query tile repeats the last visible one:
+          // the mask gives those columns an exact zero weight, the row only has to be finite.
+          const bool gathered = kGather && geo.is_global(t);
+          int rows4[4] = {0, 0, 0, 0};
+          if (gathered) {
+            const int32_t* sel = pos + geo.seg;
+            const int last = s_geo[1] - 1;                     // >= 0: there is at least one global tile
+            const int first = geo.index(t) * BN + 4 * lane;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              int64_t p = sel[min(first + k, last)];
+              if constexpr (kDebugBounds) {
+                if (p < 0 || p >= mb) {                        // a selected index names a candidate token
+                  report_bounds_ws(status, kBoundsSelectedIndex, p);
+                  p = 0;
+                }
+              }
+              rows4[k] = int(int64_t(u) * L + p);
+            }
           }
           const int slot = n % kRing;
           if (n >= kRing) {                                    // the slot's previous tile must have been consumed
@@ -279,32 +309,29 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (!ok) break;
           }
           uint64_t* full = (n == 0) ? &bars[BAR_K0_FULL] : &bars[BAR_FULL + ((n - 1) >> 1) % kPairs];
-          if (lane == 0) ptx::mbar_arrive_expect_tx(full, uint32_t(Cfg::kKV));
           uint8_t* dst = smem + Cfg::offKV + slot * Cfg::kKV;
-          if (kGather && geo.is_global(t)) {
-            // Rows 4*lane .. 4*lane+3 of the tile are the unit's selected keys number first + 4*lane ...
-            // A tile that reaches past the keys visible to this query tile repeats the last visible
-            // one: the mask gives those columns an exact zero weight, the row only has to be finite.
-            __syncwarp();                                      // the expectation is posted before any piece can land
-            const int32_t* sel = pos + geo.seg;
-            const int last = s_geo[1] - 1;                     // >= 0: there is at least one global tile
-            const int first = geo.index(t) * BN + 4 * lane;
-            int rows[4];
+          if (gathered) {
+            // A lane copies its own four rows, 16 bytes at a time, to where the 128-byte swizzle wants
+            // them: the chunk that lands at position j of the 128-byte shared-memory row r is chunk
+            // j ^ (r & 7) of the source row.
+            const uint8_t* gsrc = reinterpret_cast<const uint8_t*>(is_v ? Vraw : Kraw);
+            const uint32_t dtile = ptx::smem_u32(dst);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              int64_t p = sel[min(first + k, last)];
-              if constexpr (kDebugBounds) {
-                if (p < 0 || p >= mb) {                        // a selected index names a candidate token
-                  report_bounds_ws(status, kBoundsSelectedIndex, p);
-                  p = 0;
-                }
-              }
-              rows[k] = int(int64_t(u) * L + p);
+              const int r = 4 * lane + k;
+              const uint8_t* srow = gsrc + size_t(rows4[k]) * (D * 2);
+              const uint32_t drow = dtile + uint32_t(r) * 128u;
+              const int x = r & 7;
+#pragma unroll
+              for (int half = 0; half < Cfg::NH; ++half)
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                  ptx::cp_async_16(drow + uint32_t(half) * kHalfBytes + uint32_t(j) * 16u,
+                                   srow + half * 128 + ((j ^ x) << 4));
             }
-            for (int half = 0; half < Cfg::NH; ++half)
-              ptx::tma_gather4_2d(dst + half * kHalfBytes + lane * 512, is_v ? &map_cv : &map_ck, half * 64, rows[0],
-                                  rows[1], rows[2], rows[3], full);
+            ptx::cp_async_mbar_arrive_noinc(full);             // fires when this lane's copies have landed
           } else if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(full, uint32_t(Cfg::kKV));
             const int y = int(geo.first(t));
             for (int half = 0; half < Cfg::NH; ++half) {
               if (geo.is_global(t))
@@ -312,6 +339,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               else
                 ptx::tma_load_3d(dst + half * kHalfBytes, is_v ? &map_v : &map_k, half * 64, y, u, full);
             }
+          } else if (kGather) {
+            ptx::mbar_arrive(full);                            // a box load: the other lanes only make up the count
           }
         }
       }
@@ -566,9 +595,7 @@ bool cached_map(CUtensorMap* out, const void* base, int D, int64_t rows, int64_t
   MapEntry& slot = g_maps[g_map_next];
   g_map_next = (g_map_next + 1) % 16;
   slot.key = MapKey{nullptr, 0, 0, 0};
-  const bool encoded = heads < 0 ? encode_gather_map(&slot.map, base, D, rows)   // heads = -1: a row-gather map
-                                 : encode_map(&slot.map, base, D, rows, heads, rows);
-  if (!encoded) return false;
+  if (!encode_map(&slot.map, base, D, rows, heads, rows)) return false;
   slot.key = key;
   *out = slot.map;
   return true;
@@ -592,8 +619,9 @@ int launch_prefill_tc_impl(const tca_params* prm, const void* Q, const void* K, 
       !cached_map(&mv, V, D, L, U))
     return TCA_ERR_CUDA;
   if constexpr (kGather) {
-    if (U * L >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;   // row coordinates are 32-bit
-    if (!cached_map(&mck, K, D, U * L, -1) || !cached_map(&mcv, V, D, U * L, -1)) return TCA_ERR_CUDA;
+    if (U * L >= (int64_t(1) << 31)) return TCA_ERR_UNSUPPORTED;   // row numbers are 32-bit
+    mck = mk;   // not used by the gathering kernel
+    mcv = mv;
   } else {
     // The cache maps cover the whole flattened cache (rows past the end read as zero); a tile that
     // reaches past a unit's visible prefix reads other finite rows, which the mask turns into exact zeros.
@@ -613,7 +641,8 @@ int launch_prefill_tc_impl(const tca_params* prm, const void* Q, const void* K, 
   return launch_pdl(kern, dim3(static_cast<unsigned>(n_ctas)), dim3(kThreads), size_t(Cfg::bytes), stream, mq, mk, mv,
                     mck, mcv, pos, state, L, prm->n_q_heads, prm->n_kv_heads, prm->window, mb,
                     prm->sm_scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(O), static_cast<int*>(ws),
-                    n_qtiles, pairs, tile0, (prm->flags & TCA_FLAG_PREFILL_BAND_FIRST) ? 1 : 0);
+                    n_qtiles, pairs, tile0, (prm->flags & TCA_FLAG_PREFILL_BAND_FIRST) ? 1 : 0,
+                    static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V));
 }
 
 template <int D>

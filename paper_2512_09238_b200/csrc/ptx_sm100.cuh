@@ -140,17 +140,14 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* tmap, in
       ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
       : "memory");
 }
-// Four rows of a 2-D tensor, given by their own row coordinates, land as four consecutive rows of
-// the box (tile::gather4; the map's box is one row high).  Swizzling follows the shared-memory
-// address, so four-row pieces written at multiples of 512 bytes build the same 128-byte-swizzled
-// tile that one 128-row box load would.
-__device__ __forceinline__ void tma_gather4_2d(void* smem_dst, const void* tmap, int x, int r0, int r1, int r2,
-                                               int r3, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
-      : "memory");
+// 16 bytes from global to shared memory without a register in between (L2 only), and the arrival on
+// an mbarrier that fires once all such copies this thread has issued so far have landed; the
+// arrival counts as one of the barrier's expected arrivals (noinc).
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");

@@ -39,18 +39,4 @@ inline bool encode_map(CUtensorMap* out, const void* base, int D, int64_t rows, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The same matrix for row gathers (tile::gather4): rank 2, a box of one row x 64 columns; an
-// instruction names four rows and fills four consecutive rows of the swizzled tile.
-inline bool encode_gather_map(CUtensorMap* out, const void* base, int D, int64_t rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {cuuint64_t(D), cuuint64_t(rows > 0 ? rows : 1)};
-  cuuint64_t strides[1] = {cuuint64_t(D) * 2};
-  cuuint32_t box[2] = {64, 1};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace tca
